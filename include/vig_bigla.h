@@ -1,0 +1,128 @@
+/*
+ * vig_bigla.h -- C ABI of the B200 (sm_100a) BiGLA forward library.
+ *
+ * BiGLA is the bidirectional gated-linear-attention token mixer of ViG
+ * (arXiv 2405.18425, Sec. 4.2.1, Eq. 6).  For every (batch, head) unit, with
+ * zero initial states,
+ *
+ *     S>_t = diag(alpha>_t) S>_{t-1} + k_t^T v_t        (t = 1 .. L)
+ *     S<_t = diag(alpha<_t) S<_{t+1} + k_t^T v_t        (t = L .. 1)
+ *     out_t = ( q_t S>_t + q_t S<_t ) / 2
+ *
+ * where S is dk x dv and the gate alpha_t in (0,1]^dk scales the rows of S
+ * (G_t = alpha_t^T 1, Eq. 5).  Gates are passed as natural logarithms,
+ * log alpha = logsigmoid(g) / tau (Eq. 5 line 1 / Eq. 6 line 1, tau = 16 in the
+ * paper), which vig_gate_prep_* computes from the gate logits g.
+ *
+ * Conventions shared by every entry point
+ *   - All tensors are dense, row-major [B, H, L, d] (d = dk for q, k, g and
+ *     log alpha; d = dv for v and out): each (b, h) unit owns one contiguous
+ *     [L, d] slab.  Flattening the H x W patch grid to L is the caller's job.
+ *   - One element type per call for every tensor: bfloat16 (entry points named
+ *     *_bf16) or float (entry points named *_f32).  Accumulation is fp32.
+ *   - Unless a name says "host", every pointer is a DEVICE pointer, 16-byte
+ *     aligned, owned by the caller.  Inputs are never written; `out` is fully
+ *     overwritten.  q is used as given (no dk^-0.5 inside).
+ *   - Domain of log alpha: finite and <= 0.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Device entry points enqueue work on it and return without
+ *     synchronising.  The device of the current CUDA context must own the
+ *     buffers.
+ *   - Every entry point returns a vig_status.  Arguments are validated before
+ *     anything is launched; an invalid call launches nothing.  B, H or L equal
+ *     to 0 is a valid empty call (VIG_OK, nothing launched).
+ *   - No entry point throws, prints, or falls back to the CPU.
+ */
+#ifndef VIG_BIGLA_H
+#define VIG_BIGLA_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum vig_status {
+    VIG_OK = 0,
+    VIG_ERR_NULL_POINTER = -1,   /* a required pointer is NULL                                 */
+    VIG_ERR_BAD_DIM = -2,        /* a negative size, dk or dv < 1, tau <= 0 or not finite      */
+    VIG_ERR_UNSUPPORTED = -3,    /* dk / dv / size outside the supported set (see each call)   */
+    VIG_ERR_MISALIGNED = -4,     /* a pointer is not 16-byte aligned                            */
+    VIG_ERR_CUDA = -5,           /* a CUDA runtime call or launch failed                        */
+    VIG_ERR_WORKSPACE = -6,      /* caller-provided workspace missing or too small              */
+    VIG_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait gave up (see vig_last_device_status) */
+} vig_status;
+
+typedef enum vig_dtype { VIG_DTYPE_F32 = 0, VIG_DTYPE_BF16 = 1 } vig_dtype;
+
+/* ---- BiGLA forward (Eq. 6), device buffers ---------------------------------------------------
+ * q, k, log_alpha_fwd, log_alpha_bwd: [B,H,L,dk];  v, out: [B,H,L,dv].
+ *
+ * bf16: dk in {16, 24, 32, 64} with dv in {32, 48, 64, 128} run on the tensor-core kernels; any
+ *       other dk <= 128, dv <= 256 runs on the fp32 SIMT recurrence kernel (slow, same result
+ *       contract).  Tensor-core operands are bf16 with fp32 accumulation; the running states
+ *       stay on chip in fp32.  A unit whose gates decay by more than e^-60 inside one 16-token
+ *       block is computed by the exact in-kernel recurrence instead of the factorised tiles.
+ * f32:  dk <= 128, dv <= 256; fp32 SIMT recurrence, meant for validation-sized inputs.
+ * Long sequences are split into segments whose boundary states go through scratch memory that
+ * the library allocates and frees on `stream` (cudaMallocAsync); use the *_ws form to supply it.
+ * Errors: NULL_POINTER, BAD_DIM, UNSUPPORTED, MISALIGNED, CUDA. */
+int vig_bigla_fwd_bf16(const void* q, const void* k, const void* v,
+                       const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
+                       int B, int H, int L, int dk, int dv, void* stream);
+int vig_bigla_fwd_f32(const void* q, const void* k, const void* v,
+                      const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
+                      int B, int H, int L, int dk, int dv, void* stream);
+/* Same call as vig_bigla_fwd_bf16 (bf16 in, fp32 accumulate, bf16 out). */
+int vig_bigla_fwd(const void* q, const void* k, const void* v,
+                  const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
+                  int B, int H, int L, int dk, int dv, void* stream);
+
+/* Bytes of device scratch a vig_bigla_fwd_* call of this shape needs (0 when the whole sequence
+ * of a unit is handled by one thread block).  Returns 0 for invalid or unsupported shapes too. */
+size_t vig_bigla_workspace_bytes(int B, int H, int L, int dk, int dv, int dtype);
+/* vig_bigla_fwd_bf16 with caller-owned scratch: `ws` is a 256-byte aligned device buffer of at
+ * least vig_bigla_workspace_bytes(...) bytes (may be NULL when that is 0).  Nothing is allocated.
+ * Calls that share one `ws` must not overlap on the GPU.  Extra error: WORKSPACE. */
+int vig_bigla_fwd_ws_bf16(const void* q, const void* k, const void* v,
+                          const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
+                          int B, int H, int L, int dk, int dv,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/* ---- Gate preparation (Eq. 5 line 1 / Eq. 6 lines 1-2 after the projection) ---------------------
+ * log_alpha_x = logsigmoid(g_x) / tau for both directions, element-wise, evaluated in fp32 as
+ * (min(g,0) - log1p(exp(-|g|))) / tau and rounded to the element type.  g_*, log_alpha_*:
+ * [B,H,L,dk]; any dk >= 1; tau > 0.  In-place (log_alpha_x == g_x) is allowed.
+ * Errors: NULL_POINTER, BAD_DIM, MISALIGNED, CUDA. */
+int vig_gate_prep_bf16(const void* g_fwd, const void* g_bwd,
+                       void* log_alpha_fwd, void* log_alpha_bwd,
+                       int B, int H, int L, int dk, float tau, void* stream);
+int vig_gate_prep_f32(const void* g_fwd, const void* g_bwd,
+                      void* log_alpha_fwd, void* log_alpha_bwd,
+                      int B, int H, int L, int dk, float tau, void* stream);
+
+/* ---- Whole path on HOST buffers -------------------------------------------------------------------
+ * Gate preparation followed by the BiGLA forward (Eq. 5 line 1 + Eq. 6) for callers whose data
+ * lives in host memory.  All seven pointers are HOST pointers (pinned memory makes the copies
+ * asynchronous and faster; pageable memory works).  The call copies q, k, v, g_fwd, g_bwd to
+ * device memory it allocates on `stream`, runs both kernels there, copies `out` back, frees the
+ * device memory and synchronises `stream` before returning, so `out` is valid on return.
+ * `dtype` is a vig_dtype.  Errors: as the device calls, plus CUDA for allocation failures. */
+int vig_bigla_fwd_host(const void* q, const void* k, const void* v,
+                       const void* g_fwd, const void* g_bwd, void* out,
+                       int B, int H, int L, int dk, int dv, float tau, int dtype, void* stream);
+
+/* ---- Diagnostics ---------------------------------------------------------------------------------- */
+/* Static, NUL-terminated description of a vig_status value. */
+const char* vig_status_string(int status);
+/* Synchronises `stream`, then reads and clears the device status word of the current device.
+ * Returns VIG_OK, VIG_ERR_DEVICE_TIMEOUT if a kernel's bounded wait on an asynchronous copy
+ * expired (that unit's output is then undefined), or VIG_ERR_CUDA. */
+int vig_last_device_status(void* stream);
+/* Number of kernels this library has launched in this process so far (all devices, all streams). */
+unsigned long long vig_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VIG_BIGLA_H */

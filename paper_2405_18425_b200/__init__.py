@@ -1,0 +1,25 @@
+"""B200-native forward pass of ViG's bidirectional gated linear attention (BiGLA) token mixer.
+
+The compute lives in hand-written sm_100a CUDA kernels behind a C ABI (include/vig_bigla.h,
+libvig_bigla.so); `binding` marshals torch tensors into those calls and `synth` draws the seeded
+synthetic inputs of the benchmark configurations.  Importing the package does not load the CUDA
+library; the first binding call does and raises if it has not been built.
+"""
+from . import synth  # noqa: F401
+from .binding import (  # noqa: F401
+    VIG_DTYPE_BF16,
+    VIG_DTYPE_F32,
+    VigError,
+    load,
+    status_string,
+    vig_bigla_fwd,
+    vig_bigla_fwd_bf16,
+    vig_bigla_fwd_f32,
+    vig_bigla_fwd_host,
+    vig_bigla_fwd_ws_bf16,
+    vig_bigla_workspace_bytes,
+    vig_gate_prep_bf16,
+    vig_gate_prep_f32,
+    vig_kernel_launch_count,
+    vig_last_device_status,
+)

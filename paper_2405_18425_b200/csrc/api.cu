@@ -1,0 +1,211 @@
+// C-ABI entry points of libvig_bigla: argument validation, dispatch, host-buffer path, diagnostics.
+#include <atomic>
+#include <cmath>
+
+#include "vig_internal.h"
+
+namespace vig {
+
+__device__ int g_device_status = 0;
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int* device_status_ptr() {
+    int* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shared checks of the forward entry points.  Returns VIG_OK with *empty = true for B*H*L == 0.
+static int check_fwd_args(const void* q, const void* k, const void* v, const void* la_f, const void* la_b,
+                          const void* out, int B, int H, int L, int dk, int dv, bool* empty) {
+    *empty = false;
+    if (!q || !k || !v || !la_f || !la_b || !out) return VIG_ERR_NULL_POINTER;
+    if (B < 0 || H < 0 || L < 0 || dk < 1 || dv < 1) return VIG_ERR_BAD_DIM;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(la_f) || !aligned16(la_b) || !aligned16(out))
+        return VIG_ERR_MISALIGNED;
+    if ((long long)B * H > 0x7fffffffLL) return VIG_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0 || L == 0) *empty = true;
+    return VIG_OK;
+}
+
+static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void* la_f, const void* la_b, void* out,
+                         int B, int H, int L, int dk, int dv, void* ws, size_t ws_bytes, bool own_ws,
+                         cudaStream_t stream) {
+    bool empty;
+    int st = check_fwd_args(q, k, v, la_f, la_b, out, B, H, L, dk, dv, &empty);
+    if (st != VIG_OK) return st;
+    const long long units = (long long)B * H;
+    using bf = __nv_bfloat16;
+    const bf *q_ = (const bf*)q, *k_ = (const bf*)k, *v_ = (const bf*)v, *f_ = (const bf*)la_f, *b_ = (const bf*)la_b;
+    if (mma_supported(dk, dv)) {
+        const size_t need = mma_workspace_bytes(units, L, dk, dv);
+        if (!own_ws && need > 0) {
+            if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return VIG_ERR_WORKSPACE;
+        }
+        if (empty) return VIG_OK;
+        void* scratch = ws;
+        if (own_ws && need > 0) {
+            if (cudaMallocAsync(&scratch, need, stream) != cudaSuccess) return VIG_ERR_CUDA;
+        }
+        cudaError_t e = launch_bigla_mma(q_, k_, v_, f_, b_, (bf*)out, units, L, dk, dv, scratch, stream);
+        if (own_ws && need > 0) {
+            if (cudaFreeAsync(scratch, stream) != cudaSuccess) return VIG_ERR_CUDA;
+        }
+        return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+    }
+    if (!recurrence_supported(dk, dv)) return VIG_ERR_UNSUPPORTED;
+    if (empty) return VIG_OK;
+    cudaError_t e = launch_recurrence<bf>(q_, k_, v_, f_, b_, (bf*)out, units, L, dk, dv, stream);
+    return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
+static int fwd_f32_impl(const void* q, const void* k, const void* v, const void* la_f, const void* la_b, void* out,
+                        int B, int H, int L, int dk, int dv, cudaStream_t stream) {
+    bool empty;
+    int st = check_fwd_args(q, k, v, la_f, la_b, out, B, H, L, dk, dv, &empty);
+    if (st != VIG_OK) return st;
+    if (!recurrence_supported(dk, dv)) return VIG_ERR_UNSUPPORTED;
+    if (empty) return VIG_OK;
+    cudaError_t e = launch_recurrence<float>((const float*)q, (const float*)k, (const float*)v, (const float*)la_f,
+                                             (const float*)la_b, (float*)out, (long long)B * H, L, dk, dv, stream);
+    return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
+static int check_gate_args(const void* g_f, const void* g_b, const void* la_f, const void* la_b, int B, int H, int L,
+                           int dk, float tau, bool* empty) {
+    *empty = false;
+    if (!g_f || !g_b || !la_f || !la_b) return VIG_ERR_NULL_POINTER;
+    if (B < 0 || H < 0 || L < 0 || dk < 1 || !(tau > 0.f) || !std::isfinite(tau)) return VIG_ERR_BAD_DIM;
+    if (!aligned16(g_f) || !aligned16(g_b) || !aligned16(la_f) || !aligned16(la_b)) return VIG_ERR_MISALIGNED;
+    if (B == 0 || H == 0 || L == 0) *empty = true;
+    return VIG_OK;
+}
+
+template <typename T>
+static int gate_prep_impl(const void* g_f, const void* g_b, void* la_f, void* la_b, int B, int H, int L, int dk,
+                          float tau, cudaStream_t stream) {
+    bool empty;
+    int st = check_gate_args(g_f, g_b, la_f, la_b, B, H, L, dk, tau, &empty);
+    if (st != VIG_OK || empty) return st;
+    const long long n = (long long)B * H * L * dk;
+    cudaError_t e = launch_gate_prep<T>((const T*)g_f, (const T*)g_b, (T*)la_f, (T*)la_b, n, tau, stream);
+    return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
+}  // namespace vig
+
+using namespace vig;
+
+extern "C" {
+
+int vig_bigla_fwd_bf16(const void* q, const void* k, const void* v, const void* log_alpha_fwd,
+                       const void* log_alpha_bwd, void* out, int B, int H, int L, int dk, int dv, void* stream) {
+    return fwd_bf16_impl(q, k, v, log_alpha_fwd, log_alpha_bwd, out, B, H, L, dk, dv, nullptr, 0, true,
+                         (cudaStream_t)stream);
+}
+
+int vig_bigla_fwd(const void* q, const void* k, const void* v, const void* log_alpha_fwd, const void* log_alpha_bwd,
+                  void* out, int B, int H, int L, int dk, int dv, void* stream) {
+    return vig_bigla_fwd_bf16(q, k, v, log_alpha_fwd, log_alpha_bwd, out, B, H, L, dk, dv, stream);
+}
+
+int vig_bigla_fwd_f32(const void* q, const void* k, const void* v, const void* log_alpha_fwd,
+                      const void* log_alpha_bwd, void* out, int B, int H, int L, int dk, int dv, void* stream) {
+    return fwd_f32_impl(q, k, v, log_alpha_fwd, log_alpha_bwd, out, B, H, L, dk, dv, (cudaStream_t)stream);
+}
+
+size_t vig_bigla_workspace_bytes(int B, int H, int L, int dk, int dv, int dtype) {
+    if (B <= 0 || H <= 0 || L <= 0 || dk < 1 || dv < 1 || dtype != VIG_DTYPE_BF16) return 0;
+    if (!mma_supported(dk, dv)) return 0;
+    return mma_workspace_bytes((long long)B * H, L, dk, dv);
+}
+
+int vig_bigla_fwd_ws_bf16(const void* q, const void* k, const void* v, const void* log_alpha_fwd,
+                          const void* log_alpha_bwd, void* out, int B, int H, int L, int dk, int dv, void* ws,
+                          size_t ws_bytes, void* stream) {
+    return fwd_bf16_impl(q, k, v, log_alpha_fwd, log_alpha_bwd, out, B, H, L, dk, dv, ws, ws_bytes, false,
+                         (cudaStream_t)stream);
+}
+
+int vig_gate_prep_bf16(const void* g_fwd, const void* g_bwd, void* log_alpha_fwd, void* log_alpha_bwd, int B, int H,
+                       int L, int dk, float tau, void* stream) {
+    return gate_prep_impl<__nv_bfloat16>(g_fwd, g_bwd, log_alpha_fwd, log_alpha_bwd, B, H, L, dk, tau,
+                                         (cudaStream_t)stream);
+}
+
+int vig_gate_prep_f32(const void* g_fwd, const void* g_bwd, void* log_alpha_fwd, void* log_alpha_bwd, int B, int H,
+                      int L, int dk, float tau, void* stream) {
+    return gate_prep_impl<float>(g_fwd, g_bwd, log_alpha_fwd, log_alpha_bwd, B, H, L, dk, tau, (cudaStream_t)stream);
+}
+
+int vig_bigla_fwd_host(const void* q, const void* k, const void* v, const void* g_fwd, const void* g_bwd, void* out,
+                       int B, int H, int L, int dk, int dv, float tau, int dtype, void* stream_) {
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (!q || !k || !v || !g_fwd || !g_bwd || !out) return VIG_ERR_NULL_POINTER;
+    if (B < 0 || H < 0 || L < 0 || dk < 1 || dv < 1 || !(tau > 0.f) || !std::isfinite(tau)) return VIG_ERR_BAD_DIM;
+    if (dtype != VIG_DTYPE_F32 && dtype != VIG_DTYPE_BF16) return VIG_ERR_UNSUPPORTED;
+    if (dtype == VIG_DTYPE_F32 ? !recurrence_supported(dk, dv) : !(mma_supported(dk, dv) || recurrence_supported(dk, dv)))
+        return VIG_ERR_UNSUPPORTED;
+    if (B == 0 || H == 0 || L == 0) return VIG_OK;
+    const size_t es = dtype == VIG_DTYPE_F32 ? 4 : 2;
+    const size_t tok = (size_t)B * H * L;
+    // every slab is rounded up to 256 bytes so that all device pointers stay aligned
+    const size_t nk = (tok * dk * es + 255) / 256 * 256, nv = (tok * dv * es + 255) / 256 * 256;
+    char* base = nullptr;
+    if (cudaMallocAsync((void**)&base, 4 * nk + 2 * nv, stream) != cudaSuccess) return VIG_ERR_CUDA;
+    char *dq = base, *dk_ = base + nk, *dgf = base + 2 * nk, *dgb = base + 3 * nk, *dv_ = base + 4 * nk,
+         *dout = base + 4 * nk + nv;
+    int st = VIG_OK;
+    bool ok = cudaMemcpyAsync(dq, q, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dk_, k, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dv_, v, tok * dv * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dgf, g_fwd, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              cudaMemcpyAsync(dgb, g_bwd, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) st = VIG_ERR_CUDA;
+    if (st == VIG_OK) {
+        st = dtype == VIG_DTYPE_F32 ? vig_gate_prep_f32(dgf, dgb, dgf, dgb, B, H, L, dk, tau, stream_)
+                                    : vig_gate_prep_bf16(dgf, dgb, dgf, dgb, B, H, L, dk, tau, stream_);
+    }
+    if (st == VIG_OK) {
+        st = dtype == VIG_DTYPE_F32 ? vig_bigla_fwd_f32(dq, dk_, dv_, dgf, dgb, dout, B, H, L, dk, dv, stream_)
+                                    : vig_bigla_fwd_bf16(dq, dk_, dv_, dgf, dgb, dout, B, H, L, dk, dv, stream_);
+    }
+    if (st == VIG_OK && cudaMemcpyAsync(out, dout, tok * dv * es, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        st = VIG_ERR_CUDA;
+    if (cudaFreeAsync(base, stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
+    return st;
+}
+
+const char* vig_status_string(int status) {
+    switch (status) {
+        case VIG_OK: return "ok";
+        case VIG_ERR_NULL_POINTER: return "a required pointer is NULL";
+        case VIG_ERR_BAD_DIM: return "invalid size (negative dimension, dk or dv < 1, or tau not positive and finite)";
+        case VIG_ERR_UNSUPPORTED: return "shape or dtype outside the supported set";
+        case VIG_ERR_MISALIGNED: return "a pointer is not 16-byte aligned";
+        case VIG_ERR_CUDA: return "a CUDA runtime call or kernel launch failed";
+        case VIG_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case VIG_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int vig_last_device_status(void* stream) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return VIG_ERR_CUDA;
+    int word = 0;
+    if (cudaMemcpyFromSymbol(&word, g_device_status, sizeof(int)) != cudaSuccess) return VIG_ERR_CUDA;
+    if (word != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return VIG_ERR_CUDA;
+    }
+    return (word & kDevStatusTimeout) ? VIG_ERR_DEVICE_TIMEOUT : VIG_OK;
+}
+
+unsigned long long vig_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

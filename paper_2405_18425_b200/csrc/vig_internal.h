@@ -1,0 +1,36 @@
+// Internal declarations shared by the translation units of libvig_bigla (not part of the C ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "vig_bigla.h"
+
+namespace vig {
+
+// Device status word: bit flags set by kernels whose bounded waits expire.
+constexpr int kDevStatusTimeout = 1;
+int* device_status_ptr();            // device address of the status word of the current device (NULL on error)
+void count_launch(unsigned n = 1);   // bumps the process-wide launch counter
+
+// ---- fp32 SIMT recurrence (Eq. 6 evaluated step by step), any dk <= 128, dv <= 256 ----
+bool recurrence_supported(int dk, int dv);
+template <typename T>
+cudaError_t launch_recurrence(const T* q, const T* k, const T* v, const T* la_f, const T* la_b, T* out,
+                              long long units, int L, int dk, int dv, cudaStream_t stream);
+
+// ---- gate preparation ----
+template <typename T>
+cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long long n, float tau,
+                             cudaStream_t stream);
+
+// ---- bf16 tensor-core path ----
+bool mma_supported(int dk, int dv);
+// Scratch bytes needed for the segmented (long-L) path; 0 if one thread block covers a unit.
+size_t mma_workspace_bytes(long long units, int L, int dk, int dv);
+cudaError_t launch_bigla_mma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                             const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
+                             long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
+
+}  // namespace vig

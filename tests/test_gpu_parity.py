@@ -1,0 +1,275 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded
+inputs.  Bar: max|gpu - oracle| <= 1e-4 * max|oracle| for fp32 storage and <= 2e-2 * max|oracle|
+for bf16 storage, the maximum taken over the whole output tensor."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2405_18425_b200 as vig
+from paper_2405_18425_b200 import synth
+
+from helpers import (TOL, device_to_f64, oracle_log_alpha, oracle_out, random_problem, rel_err, to_device,
+                     to_stored)
+
+pytestmark = pytest.mark.gpu
+
+
+def _fwd(dtype):
+    return vig.vig_bigla_fwd_f32 if dtype == "f32" else vig.vig_bigla_fwd_bf16
+
+
+def _run_unfused(oracle, cfg, x):
+    """Oracle gate prep -> stored log alpha (same bytes for both sides) -> GPU forward vs oracle forward."""
+    la_f = oracle_log_alpha(oracle, x["g_fwd"], cfg.dtype, cfg.tau)
+    la_b = oracle_log_alpha(oracle, x["g_bwd"], cfg.dtype, cfg.tau)
+    d = {n: to_device(a, cfg.dtype) for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    out = torch.empty_like(d["v"])
+    _fwd(cfg.dtype)(d["q"], d["k"], d["v"], d["f"], d["b"], out)
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    ref = oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, cfg.dtype)
+    return device_to_f64(out, cfg.dtype), ref
+
+
+@pytest.mark.parametrize("idx", range(len(synth.CONFIGS)), ids=[c.name for c in synth.CONFIGS])
+def test_benchmark_config_full_size(oracle, idx):
+    """All five configurations at full size, every output element compared."""
+    cfg = synth.CONFIGS[idx]
+    got, ref = _run_unfused(oracle, cfg, synth.make_inputs(cfg))
+    assert np.isfinite(got).all()
+    assert rel_err(got, ref) <= TOL[cfg.dtype]
+
+
+@pytest.mark.parametrize("dk,dv", [(16, 32), (24, 48), (32, 64), (64, 128), (16, 48), (8, 16), (40, 72)])
+@pytest.mark.parametrize("L", [1, 5, 16, 17, 33, 100, 250])
+def test_bf16_small_and_ragged(oracle, dk, dv, L):
+    """Lengths below, at and across the 16-token tile, several head sizes (the last two are not on
+    the tensor-core path and exercise the SIMT recurrence kernel through the same entry point)."""
+    cfg, x = random_problem(100 + L, 2, 3, L, dk, dv, "bf16")
+    got, ref = _run_unfused(oracle, cfg, x)
+    assert rel_err(got, ref) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("dk,dv,L", [(16, 32, 7), (16, 32, 130), (24, 48, 50), (5, 3, 33), (128, 256, 20),
+                                     (32, 64, 600)])
+def test_f32_shapes(oracle, dk, dv, L):
+    cfg, x = random_problem(200 + L, 2, 2, L, dk, dv, "f32")
+    got, ref = _run_unfused(oracle, cfg, x)
+    assert rel_err(got, ref) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("L", [600, 2049, 4096 + 37])
+def test_bf16_long_sequences(oracle, L):
+    """Sequences split into several segments with a ragged last segment."""
+    cfg, x = random_problem(300 + L, 1, 3, L, 24, 48, "bf16")
+    got, ref = _run_unfused(oracle, cfg, x)
+    assert rel_err(got, ref) <= TOL["bf16"]
+    cfg, x = random_problem(301 + L, 1, 2, L, 32, 64, "bf16", gate_mean=2.0)
+    got, ref = _run_unfused(oracle, cfg, x)
+    assert rel_err(got, ref) <= TOL["bf16"]
+
+
+def _gate_cases(L, dk, rng):
+    zero = np.zeros((1, 1, L, dk))
+    closed = np.full((1, 1, L, dk), -1.0e3)
+    wall = zero.copy()
+    wall[0, 0, L // 2] = -1.0e3
+    mixed = -rng.random((1, 1, L, dk)) * np.where(rng.random((1, 1, L, dk)) < 0.1, 40.0, 0.05)
+    steep = np.full((1, 1, L, dk), -6.0)            # decays by e^-96 inside a 16-token block
+    return {"alpha_one": zero, "closed": closed, "wall": wall, "mixed": mixed, "steep": steep}
+
+
+@pytest.mark.parametrize("case", ["alpha_one", "closed", "wall", "mixed", "steep"])
+@pytest.mark.parametrize("dtype,dk,dv,L", [("bf16", 32, 64, 196), ("bf16", 24, 48, 700), ("f32", 16, 32, 64)])
+def test_degenerate_gates(oracle, case, dtype, dk, dv, L):
+    """alpha == 1 (plain linear attention), fully closed gates (only the s = t term survives), a single
+    closed gate, and gates mixing slow decay with hard resets: the result must stay finite and match."""
+    rng = np.random.default_rng(7)
+    cfg, x = random_problem(400, 1, 2, L, dk, dv, dtype)
+    la = [np.broadcast_to(_gate_cases(L, dk, rng)[case], (1, 2, L, dk)) for _ in range(2)]
+    la_f, la_b = synth.store(la[0], dtype), synth.store(la[1], dtype)
+    d = {n: to_device(a, dtype) for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    out = torch.empty_like(d["v"])
+    _fwd(dtype)(d["q"], d["k"], d["v"], d["f"], d["b"], out)
+    torch.cuda.synchronize()
+    got = device_to_f64(out, dtype)
+    ref = oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, dtype)
+    assert np.isfinite(got).all()
+    assert rel_err(got, ref) <= TOL[dtype]
+    if case == "closed":
+        f = lambda n: synth.stored_to_f64(x[n], dtype)
+        diag = np.einsum("bhti,bhti->bht", f("q"), f("k"))[..., None] * f("v")
+        assert rel_err(got, diag) <= TOL[dtype]
+
+
+def test_mixed_units_fast_and_exact_paths(oracle):
+    """One unit with out-of-range gates among ordinary units must not disturb its neighbours."""
+    cfg, x = random_problem(500, 2, 3, 196, 32, 64, "bf16")
+    la_f = synth.stored_to_f64(oracle_log_alpha(oracle, x["g_fwd"], "bf16", 16.0), "bf16")
+    la_b = synth.stored_to_f64(oracle_log_alpha(oracle, x["g_bwd"], "bf16", 16.0), "bf16")
+    la_f[1, 0, 40:60] = -7.0
+    la_b[0, 2, 100:101] = -90.0
+    la_f, la_b = synth.store(la_f, "bf16"), synth.store(la_b, "bf16")
+    d = {n: to_device(a, "bf16") for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    out = torch.empty_like(d["v"])
+    vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], out)
+    got = device_to_f64(out, "bf16")
+    ref = oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, "bf16")
+    assert rel_err(got, ref) <= TOL["bf16"]
+    for b in range(2):
+        for h in range(3):
+            assert rel_err(got[b, h], ref[b, h]) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gate_prep_matches_oracle(oracle, dtype):
+    r = np.random.default_rng(3)
+    g = np.concatenate([r.standard_normal(5000) * 3.0, np.array([0.0, -0.0, 50.0, -50.0, 88.0, -88.0, 200.0, -200.0,
+                                                                  1e-3, -1e-3]), r.standard_normal(6) * 30.0])
+    g = np.resize(g, (2, 3, 19, 44))                       # n = 5016 elements: vector body and scalar tail
+    gs = synth.store(g, dtype)
+    for tau in (16.0, 1.0, 3.0):
+        gf, gb = to_device(gs, dtype), to_device(synth.store(-g, dtype), dtype)
+        of, ob = torch.empty_like(gf), torch.empty_like(gb)
+        fn = vig.vig_gate_prep_f32 if dtype == "f32" else vig.vig_gate_prep_bf16
+        fn(gf, gb, of, ob, tau)
+        torch.cuda.synchronize()
+        for got_t, g_in in ((of, gs), (ob, synth.store(-g, dtype))):
+            ref = oracle.gate_prep(synth.stored_to_f64(g_in, dtype), tau)
+            got = device_to_f64(got_t, dtype)
+            assert np.isfinite(got).all() and (got <= 0).all()
+            # fp32 evaluation then rounding to storage: a few fp32 ulps, plus one storage ulp for bf16
+            ulp = 2.0 ** -22 if dtype == "f32" else 2.0 ** -8
+            assert np.all(np.abs(got - ref) <= ulp * np.abs(ref) + 1e-37)
+    # in place
+    gf = to_device(gs, dtype)
+    keep = gf.clone()
+    o2 = torch.empty_like(gf)
+    fn(keep, keep.clone(), o2, torch.empty_like(gf), 16.0)
+    gb = gf.clone()
+    fn(gf, gb, gf, gb, 16.0)
+    assert torch.equal(gf, o2)
+
+
+def test_whole_path_gate_prep_then_forward(oracle):
+    """GPU gate prep feeding the GPU forward, against the oracle chain from the same logits (the
+    oracle keeps log alpha in fp64, the un-fused GPU path rounds it to bf16 in between)."""
+    cfg = synth.CONFIGS[3]
+    x = synth.make_inputs(cfg, units=slice(0, 24))
+    d = {n: to_device(a, cfg.dtype) for n, a in x.items()}
+    la_f, la_b = torch.empty_like(d["g_fwd"]), torch.empty_like(d["g_bwd"])
+    vig.vig_gate_prep_bf16(d["g_fwd"], d["g_bwd"], la_f, la_b, cfg.tau)
+    out = torch.empty_like(d["v"])
+    vig.vig_bigla_fwd(d["q"], d["k"], d["v"], la_f, la_b, out)
+    f = lambda n: synth.stored_to_f64(x[n], cfg.dtype)
+    ref = oracle.bigla_fwd(f("q"), f("k"), f("v"), oracle.gate_prep(f("g_fwd"), cfg.tau),
+                           oracle.gate_prep(f("g_bwd"), cfg.tau), nthreads=8)
+    assert rel_err(device_to_f64(out, cfg.dtype), ref) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("idx", [0, 3, 4])
+def test_host_entry_point_matches_device_path(oracle, idx):
+    cfg = synth.CONFIGS[idx]
+    n_units = min(cfg.units, 16)
+    x = synth.make_inputs(cfg, units=slice(0, n_units))
+    host = {n: torch.from_numpy(a.view(np.int16) if cfg.dtype == "bf16" else a).pin_memory() for n, a in x.items()}
+    out_h = torch.empty(x["v"].shape, dtype=host["v"].dtype).pin_memory()
+    code = vig.VIG_DTYPE_F32 if cfg.dtype == "f32" else vig.VIG_DTYPE_BF16
+    vig.vig_bigla_fwd_host(host["q"], host["k"], host["v"], host["g_fwd"], host["g_bwd"], out_h, cfg.tau, code)
+    d = {n: to_device(a, cfg.dtype) for n, a in x.items()}
+    la_f, la_b = torch.empty_like(d["g_fwd"]), torch.empty_like(d["g_bwd"])
+    (vig.vig_gate_prep_f32 if cfg.dtype == "f32" else vig.vig_gate_prep_bf16)(d["g_fwd"], d["g_bwd"], la_f, la_b, cfg.tau)
+    out_d = torch.empty_like(d["v"])
+    _fwd(cfg.dtype)(d["q"], d["k"], d["v"], la_f, la_b, out_d)
+    torch.cuda.synchronize()
+    ref_bytes = to_stored(out_d, cfg.dtype)
+    got_bytes = out_h.numpy().view(np.uint16) if cfg.dtype == "bf16" else out_h.numpy()
+    np.testing.assert_array_equal(got_bytes, ref_bytes)
+    # and numpy arrays (pageable memory) work as well
+    out_n = np.empty_like(x["v"])
+    vig.vig_bigla_fwd_host(x["q"], x["k"], x["v"], x["g_fwd"], x["g_bwd"], out_n, cfg.tau, code)
+    np.testing.assert_array_equal(out_n, ref_bytes)
+
+
+def test_workspace_variant_and_determinism(oracle):
+    cfg = synth.CONFIGS[4]
+    x = synth.make_inputs(cfg, units=slice(0, 6))
+    la_f = oracle_log_alpha(oracle, x["g_fwd"], "bf16", 16.0)
+    la_b = oracle_log_alpha(oracle, x["g_bwd"], "bf16", 16.0)
+    d = {n: to_device(a, "bf16") for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    need = vig.vig_bigla_workspace_bytes(6, 1, cfg.L, cfg.dk, cfg.dv)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    outs = []
+    for _ in range(2):
+        o = torch.full_like(d["v"], float("nan"))
+        vig.vig_bigla_fwd_ws_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], o, ws)
+        outs.append(o)
+        o = torch.full_like(d["v"], float("nan"))
+        vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], o)
+        outs.append(o)
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        assert torch.equal(o.view(torch.int16), outs[0].view(torch.int16))     # bit-identical run to run
+    with pytest.raises(vig.VigError) as e:
+        vig.vig_bigla_fwd_ws_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], outs[0], ws[: need - 256])
+    assert e.value.status == -6
+
+
+def test_short_sequence_determinism_and_streams(oracle):
+    cfg = synth.CONFIGS[2]
+    x = synth.make_inputs(cfg, units=slice(0, 40))
+    la_f = oracle_log_alpha(oracle, x["g_fwd"], "bf16", 16.0)
+    la_b = oracle_log_alpha(oracle, x["g_bwd"], "bf16", 16.0)
+    d = {n: to_device(a, "bf16") for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    a = torch.empty_like(d["v"])
+    vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], a)
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    b = torch.full_like(d["v"], float("nan"))
+    before = vig.vig_kernel_launch_count()
+    with torch.cuda.stream(s):
+        vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], b)
+    s.synchronize()
+    assert vig.vig_kernel_launch_count() > before
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    # inputs are never written
+    for n, src in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items():
+        np.testing.assert_array_equal(to_stored(d[n], "bf16"), src)
+
+
+def test_empty_calls_on_device():
+    z = torch.empty(0, 2, 8, 16, device="cuda", dtype=torch.bfloat16)
+    zv = torch.empty(0, 2, 8, 32, device="cuda", dtype=torch.bfloat16)
+    # data_ptr() of an empty tensor is NULL, so pass a real allocation with a zero batch
+    buf = torch.empty(64, device="cuda", dtype=torch.bfloat16)
+    lib = vig.load()
+    p = buf.data_ptr()
+    assert lib.vig_bigla_fwd_bf16(p, p, p, p, p, p, 0, 2, 8, 16, 32, None) == 0
+    assert lib.vig_bigla_fwd_f32(p, p, p, p, p, p, 2, 2, 0, 16, 32, None) == 0
+    assert lib.vig_gate_prep_bf16(p, p, p, p, 2, 0, 8, 16, 16.0, None) == 0
+    assert z.numel() == 0 and zv.numel() == 0
+
+
+def test_golden_samples(oracle):
+    """Sampled outputs of every configuration stored by tests/golden/make_golden.py (oracle only;
+    gates kept in fp64 there, rounded to storage here, which the tolerance covers)."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "bigla_samples.txt")
+    rows = [ln.split() for ln in open(path) if ln.strip() and not ln.startswith("#")]
+    by_unit = {}
+    for name, u, t, j, val in rows:
+        by_unit.setdefault((name, int(u)), []).append((int(t), int(j), float(val)))
+    for (name, u), samples in by_unit.items():
+        cfg = synth.CONFIG_BY_NAME[name]
+        x = synth.make_inputs(cfg, units=slice(u, u + 1))
+        d = {n: to_device(a, cfg.dtype) for n, a in x.items()}
+        la_f, la_b = torch.empty_like(d["g_fwd"]), torch.empty_like(d["g_bwd"])
+        (vig.vig_gate_prep_f32 if cfg.dtype == "f32" else vig.vig_gate_prep_bf16)(d["g_fwd"], d["g_bwd"], la_f, la_b, cfg.tau)
+        out = torch.empty_like(d["v"])
+        _fwd(cfg.dtype)(d["q"], d["k"], d["v"], la_f, la_b, out)
+        got = device_to_f64(out, cfg.dtype)[0, 0]
+        scale = np.abs(got).max()
+        for t, j, val in samples:
+            assert abs(got[t, j] - val) <= TOL[cfg.dtype] * scale
