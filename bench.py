@@ -168,6 +168,7 @@ def run_gpu(args, cfg):
     import torch
 
     import paper_2405_18425_b200 as vig
+    from paper_2405_18425_b200 import dist as vdist
     from paper_2405_18425_b200 import synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -246,11 +247,7 @@ def run_gpu(args, cfg):
     if dist is not None:
         dist.barrier()
     launches = vig.vig_kernel_launch_count() - launches0
-    total_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = vdist.max_over_ranks(e0.elapsed_time(e1), dist, device="cuda")   # slowest rank
     ms_per_step = total_ms / args.steps
     clocks = sampler.summary(t_host0, t_host1)
 
@@ -265,7 +262,7 @@ def run_gpu(args, cfg):
     assert vig.vig_last_device_status() == 0, "a device-side bounded wait expired"
 
     tokens_per_step = cfg.tokens
-    value = world * tokens_per_step / (ms_per_step * 1e-3)
+    value = vdist.job_throughput(tokens_per_step, ms_per_step, world)
     peak, peak_kind = _peaks()
     achieved = cfg.algorithmic_bytes / (scan_us * 1e-6) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
