@@ -58,8 +58,8 @@ typedef enum vig_dtype { VIG_DTYPE_F32 = 0, VIG_DTYPE_BF16 = 1 } vig_dtype;
 /* ---- BiGLA forward (Eq. 6), device buffers ---------------------------------------------------
  * q, k, log_alpha_fwd, log_alpha_bwd: [B,H,L,dk];  v, out: [B,H,L,dv].
  *
- * bf16: dk in {16, 24, 32, 64} with dv in {32, 48, 64, 128} run on the tensor-core kernels; any
- *       other dk <= 128, dv <= 256 runs on the fp32 SIMT recurrence kernel (slow, same result
+ * bf16: dk in {16, 24, 32} with dv in {32, 48, 64} run on the tensor-core kernels; any other
+ *       dk <= 128, dv <= 256 runs on the fp32 SIMT recurrence kernel (slow, same result
  *       contract).  Tensor-core operands are bf16 with fp32 accumulation; the running states
  *       stay on chip in fp32.  A unit whose gates decay by more than e^-60 inside one 16-token
  *       block is computed by the exact in-kernel recurrence instead of the factorised tiles.
@@ -88,6 +88,31 @@ int vig_bigla_fwd_ws_bf16(const void* q, const void* k, const void* v,
                           const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
                           int B, int H, int L, int dk, int dv,
                           void* ws, size_t ws_bytes, void* stream);
+
+/* vig_bigla_fwd_bf16 for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a library convenience).  Some users of this code run where cudaMalloc is off limits at call
+ * time: a serving loop whose memory budget was fixed at start-up, a process that shares the GPU under
+ * a hard partition where a late allocation can fail or stall every stream, or an embedding
+ * application that simply hands the library no allocator.  The other entry points either allocate
+ * scratch on the stream or need a caller-made workspace; this one does neither.  Its scratch is a
+ * fixed VIG_STATIC_SCRATCH_BYTES array inside the library's device image, which every GPU that loads
+ * the library holds until the process exits.
+ *   - Only the tensor-core shapes (dk in {16,24,32}, dv in {32,48,64}); otherwise UNSUPPORTED.
+ *   - A problem whose scratch need (vig_bigla_workspace_bytes) exceeds VIG_STATIC_SCRATCH_BYTES is
+ *     rejected with VIG_ERR_WORKSPACE and nothing is launched; use vig_bigla_fwd_ws_bf16 for it.
+ *   - No cudaMalloc, cudaFree or other allocating call is made, by this entry point or beneath it.
+ *   - The first call on each device looks up the array's device address (a one-time set-up step for
+ *     that device); make that first call with the device current and before starting any stream
+ *     capture.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left in it.
+ *     The call itself clears the part that must start at zero.  Two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it and give undefined results: order them.
+ * Results are identical to vig_bigla_fwd_bf16.  Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED,
+ * WORKSPACE, CUDA. */
+#define VIG_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int vig_bigla_fwd_static_bf16(const void* q, const void* k, const void* v,
+                              const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
+                              int B, int H, int L, int dk, int dv, void* stream);
 
 /* ---- Gate preparation (Eq. 5 line 1 / Eq. 6 lines 1-2 after the projection) ---------------------
  * log_alpha_x = logsigmoid(g_x) / tau for both directions, element-wise, evaluated in fp32 as

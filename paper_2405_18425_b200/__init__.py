@@ -16,6 +16,7 @@ from .binding import (  # noqa: F401
     vig_bigla_fwd_bf16,
     vig_bigla_fwd_f32,
     vig_bigla_fwd_host,
+    vig_bigla_fwd_static_bf16,
     vig_bigla_fwd_ws_bf16,
     vig_bigla_workspace_bytes,
     vig_gate_prep_bf16,

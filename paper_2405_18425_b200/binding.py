@@ -39,7 +39,7 @@ def load() -> ctypes.CDLL:
         lib = ctypes.CDLL(LIB_PATH)
         vp, ci, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
         fwd = [vp] * 6 + [ci] * 5 + [vp]
-        for name in ("vig_bigla_fwd", "vig_bigla_fwd_bf16", "vig_bigla_fwd_f32"):
+        for name in ("vig_bigla_fwd", "vig_bigla_fwd_bf16", "vig_bigla_fwd_f32", "vig_bigla_fwd_static_bf16"):
             getattr(lib, name).argtypes = fwd
             getattr(lib, name).restype = ci
         lib.vig_bigla_fwd_ws_bf16.argtypes = [vp] * 6 + [ci] * 5 + [vp, ctypes.c_size_t, vp]
@@ -108,6 +108,15 @@ def vig_bigla_fwd_f32(q, k, v, log_alpha_fwd, log_alpha_bwd, out, stream=None):
     _check(load().vig_bigla_fwd_f32(q.data_ptr(), k.data_ptr(), v.data_ptr(), log_alpha_fwd.data_ptr(),
                                     log_alpha_bwd.data_ptr(), out.data_ptr(), *_dims(q, v), _stream(stream)),
            "vig_bigla_fwd_f32")
+    return out
+
+
+def vig_bigla_fwd_static_bf16(q, k, v, log_alpha_fwd, log_alpha_bwd, out, stream=None):
+    """The forward pass with the library's fixed built-in scratch: allocates nothing (see the header)."""
+    _dev(q, k, v, log_alpha_fwd, log_alpha_bwd, out)
+    _check(load().vig_bigla_fwd_static_bf16(q.data_ptr(), k.data_ptr(), v.data_ptr(), log_alpha_fwd.data_ptr(),
+                                            log_alpha_bwd.data_ptr(), out.data_ptr(), *_dims(q, v),
+                                            _stream(stream)), "vig_bigla_fwd_static_bf16")
     return out
 
 
