@@ -144,6 +144,17 @@ const char* vig_status_string(int status);
  * Returns VIG_OK, VIG_ERR_DEVICE_TIMEOUT if a kernel's bounded wait on an asynchronous copy
  * expired (that unit's output is then undefined), or VIG_ERR_CUDA. */
 int vig_last_device_status(void* stream);
+/* Which kernel family the bf16 forward entry points use, process-wide (a testing and profiling aid:
+ * all families compute the same function and meet the same tolerance).
+ *   VIG_KERNEL_AUTO      tcgen05/TMEM kernel where it applies (dk in {24,32}, dv in {48,64}, L <= 256),
+ *                        else the mma.sync tensor-core kernel, else the SIMT recurrence   (default)
+ *   VIG_KERNEL_MMA_SYNC  never the tcgen05 kernel
+ *   VIG_KERNEL_SIMT      always the fp32 SIMT recurrence kernel
+ * Returns VIG_OK, or VIG_ERR_UNSUPPORTED for an unknown value (the setting is then unchanged). */
+#define VIG_KERNEL_AUTO 0
+#define VIG_KERNEL_MMA_SYNC 1
+#define VIG_KERNEL_SIMT 2
+int vig_set_kernel_preference(int preference);
 /* Number of kernels this library has launched in this process so far (all devices, all streams). */
 unsigned long long vig_kernel_launch_count(void);
 

@@ -55,6 +55,8 @@ def load() -> ctypes.CDLL:
         lib.vig_status_string.restype = ctypes.c_char_p
         lib.vig_last_device_status.argtypes = [vp]
         lib.vig_last_device_status.restype = ci
+        lib.vig_set_kernel_preference.argtypes = [ci]
+        lib.vig_set_kernel_preference.restype = ci
         lib.vig_kernel_launch_count.argtypes = []
         lib.vig_kernel_launch_count.restype = ctypes.c_ulonglong
         _lib = lib
@@ -172,6 +174,13 @@ def vig_bigla_fwd_host(q, k, v, g_fwd, g_bwd, out, tau=16.0, dtype=VIG_DTYPE_BF1
 
 def vig_last_device_status(stream=None) -> int:
     return int(load().vig_last_device_status(_stream(stream)))
+
+
+VIG_KERNEL_AUTO, VIG_KERNEL_MMA_SYNC, VIG_KERNEL_SIMT = 0, 1, 2
+
+
+def vig_set_kernel_preference(preference: int) -> None:
+    _check(load().vig_set_kernel_preference(int(preference)), "vig_set_kernel_preference")
 
 
 def vig_kernel_launch_count() -> int:

@@ -9,6 +9,8 @@ namespace vig {
 __device__ int g_device_status = 0;
 
 static std::atomic<unsigned long long> g_launches{0};
+static std::atomic<int> g_kernel_pref{VIG_KERNEL_AUTO};
+int kernel_preference() { return g_kernel_pref.load(std::memory_order_relaxed); }
 void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 int* device_status_ptr() {
@@ -41,7 +43,7 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
     const long long units = (long long)B * H;
     using bf = __nv_bfloat16;
     const bf *q_ = (const bf*)q, *k_ = (const bf*)k, *v_ = (const bf*)v, *f_ = (const bf*)la_f, *b_ = (const bf*)la_b;
-    if (mma_supported(dk, dv)) {
+    if (mma_supported(dk, dv) && kernel_preference() != VIG_KERNEL_SIMT) {
         const size_t need = mma_workspace_bytes(units, L, dk, dv);
         if (!own_ws && need > 0) {
             if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return VIG_ERR_WORKSPACE;
@@ -204,6 +206,13 @@ int vig_last_device_status(void* stream) {
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return VIG_ERR_CUDA;
     }
     return (word & kDevStatusTimeout) ? VIG_ERR_DEVICE_TIMEOUT : VIG_OK;
+}
+
+int vig_set_kernel_preference(int preference) {
+    if (preference != VIG_KERNEL_AUTO && preference != VIG_KERNEL_MMA_SYNC && preference != VIG_KERNEL_SIMT)
+        return VIG_ERR_UNSUPPORTED;
+    g_kernel_pref.store(preference, std::memory_order_relaxed);
+    return VIG_OK;
 }
 
 unsigned long long vig_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
