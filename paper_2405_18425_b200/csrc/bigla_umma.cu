@@ -1,18 +1,25 @@
 // bf16 BiGLA forward on the 5th-generation tensor cores (tcgen05.mma, accumulators in TMEM).
 //
-// One thread block owns one (batch, head) unit of up to 256 tokens, split into chunks of C = 128.
-// With b_t the inclusive prefix sum of log alpha> from the start of the chunk (e_t the inclusive
-// suffix sum of log alpha< to its end), Eq. 6 becomes, per chunk,
-//     P    = tril(q~> k~>^T) + triu(q~< k~<^T)          q~> = q e^{b},  k~> = k e^{-b},  q~< = q e^{e},  k~< = k e^{-e}
-//     out  = ( P v + q~> S>_in + q~< S<_in ) / 2
-//     U    = [k~< | k~>]^T v                            (zero-input chunk summaries, both directions in one MMA)
-//     S>_in(c+1) = (S>_in(c) + U>_c) * e^{b_last}       (rows scaled; mirrored for <)
-// Every product is a tcgen05.mma with M = 128: P (N = 128, K = dk), U (A = the four operand tiles stacked
-// along M, MN-major), P v (A = bf16 P read straight from TMEM), q~ S (B = the bf16 state tile).  The
-// threads only do the element-wise work: operand scaling in place (phase 1), masking / packing P,
-// scaling the chunk summaries, and the output epilogue.  TMEM use is 256 columns, shared memory
-// 109 KB, so two blocks share an SM and one block's MMA round trips hide behind the other's
-// element-wise phases.
+// One thread block owns one (batch, head) unit of up to 256 tokens, split into chunks of C = 128
+// rows; thread r of the block owns token r (TMEM lane r mod 128 of chunk r / 128) in every
+// element-wise phase.  With b_t the inclusive prefix sum of log alpha> from the start of the chunk
+// and e_t the inclusive suffix sum of log alpha< to its end, Eq. 6 becomes, per chunk,
+//     [b | e] = T> la> | T< la<                      prefix sums as products with 0/1 triangular matrices
+//     q~> = q e^{b},  k~> = k e^{-b},  q~< = q e^{e},  k~< = k e^{-e}
+//     P    = tril(q~> k~>^T) + triu(q~< k~<^T)
+//     U    = [k~< | k~>]^T v                          zero-input chunk summaries, both directions in one product
+//     out  = ( P v + q~> S>_in + q~< S<_in ) / 2      S>_in = U>(left chunk) * e^{b_last}, mirrored for <
+// Every product is a tcgen05.mma with M = 128:
+//   - the prefix sums: A = a 128-row window of a 240-row 0/1 tile ([zeros; lower triangle; ones],
+//     shifted by 16 rows per K step), B = the log-gate tile as loaded; fp32 accumulation of bf16
+//     values times 0/1 is exact up to fp32 addition;
+//   - P in two column halves (fwd and bwd side by side in TMEM, so the mask and the sum of the
+//     diagonal block happen in fp32), packed to bf16 and written back to TMEM as the A operand of P v;
+//   - U with A = the four operand tiles stacked along M (MN-major), q~ S with B = the bf16 state tile.
+// The threads only do element-wise work on their own row: operand scaling in place, masking and
+// packing P, scaling the chunk summaries, the output epilogue.  TMEM use is 256 columns (128 per
+// chunk: prefix sums, then P, then bf16 P + U / out), shared memory about 102 KB at L = 196, so
+// two blocks share an SM and one block's MMA round trips hide behind the other's element-wise phases.
 #include <cuda.h>
 
 #include "ptx.cuh"
@@ -23,18 +30,14 @@
 namespace vig {
 namespace {
 
-constexpr int kBlk = 16;        // rows per prefix-sum block
 constexpr int kChunk = 128;     // rows per MMA chunk
-constexpr int kRows = 256;      // rows of every shared-memory tile (TMA zero-fills rows >= L)
+constexpr int kMaxRows = 256;   // longest unit this kernel takes
 constexpr int kThreads = 256;
 constexpr float kGateRange = 60.f;
 constexpr float kLog2e = 1.4426950408889634f;
-
-// TMEM column map (256 columns allocated)
-constexpr uint32_t kT1 = 0;      // P tile, fp32 [128 x 128]; later bf16 P in its first 64 columns
-constexpr uint32_t kTO = 128;    // output accumulator [128 x 64]; before that, the summary U of chunk 1
-constexpr uint32_t kTU = 192;    // summary U of chunk 0 [128 x 64]
 constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kZRows = 240;                 // 112 constant rows, 16 triangle rows, 112 constant rows
+constexpr uint32_t kZBytes = kZRows * 32;        // 16 bf16 per row
 
 // ---- tcgen05 wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -44,7 +47,7 @@ __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sy
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Shared-memory matrix descriptor (start address, leading / stride byte offsets in 16-byte units,
-// descriptor version 1, swizzle mode in bits 61..63: 2 = 128B, 4 = 64B).
+// descriptor version 1, swizzle mode in bits 61..63: 0 = none, 2 = 128B, 4 = 64B).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle) {
     return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) | ((uint64_t)1 << 46) | ((uint64_t)swizzle << 61);
@@ -69,6 +72,13 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(addr));
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -87,45 +97,112 @@ __device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]
         "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
-__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
 }
+__device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
 
-struct USmem {
-    static constexpr uint32_t a0 = 0;                          // four q-type tiles, 16 KB each
-    static constexpr uint32_t tile = kRows * 64;
-    static constexpr uint32_t v = 4 * tile;                    // v tile, later the output tile (32 KB)
-    static constexpr uint32_t s_fwd = v + kRows * 128;         // bf16 state entering chunk 1 from the left  [32 x 64]
-    static constexpr uint32_t s_bwd = s_fwd + 32 * 128;        // bf16 state entering chunk 0 from the right [32 x 64]
-    static constexpr uint32_t tot = s_bwd + 32 * 128;          // [2][16][32] fp32 block sums of log2 alpha
-    static constexpr uint32_t misc = tot + 2 * 16 * 32 * 4;    // mbarriers, TMEM slot, flag
-    static constexpr uint32_t total = misc + 64;
+// ---- shared-memory plan (rows = tokens of the unit rounded up to 16) ---------------------------
+struct ULayout {
+    uint32_t tile;     // bytes of one q-type tile [rows][32] bf16 (64-byte rows, 64B swizzle); four of them from offset 0:
+                       //   as loaded: q, k, log alpha>, log alpha<;  after scaling: k~<, k~>, q~>, q~<
+    uint32_t v;        // v tile [rows][64] bf16 (128B swizzle), later the output tile
+    uint32_t zf, zb;   // 0/1 tiles of the prefix / suffix sums
+    uint32_t s_fwd;    // bf16 state entering chunk 1 from the left  [32][64] (128B swizzle)
+    uint32_t s_bwd;    // bf16 state entering chunk 0 from the right
+    uint32_t dec;      // [2][32] fp32 chunk decay factors e^{b_last} (fwd, chunk 0), e^{e_first} (bwd, chunk 1)
+    uint32_t misc;     // mbarriers, TMEM slot, flag
+    uint32_t total;
 };
+__host__ __device__ inline ULayout make_layout(int rows) {
+    ULayout l;
+    l.tile = (uint32_t)rows * 64;
+    l.v = 4 * l.tile;
+    l.zf = l.v + (uint32_t)rows * 128;
+    l.zb = l.zf + kZBytes;
+    l.s_fwd = (l.zb + kZBytes + 1023u) & ~1023u;
+    l.s_bwd = l.s_fwd + 32 * 128;
+    l.dec = l.s_bwd + 32 * 128;
+    l.misc = l.dec + 2 * 32 * 4;
+    l.total = l.misc + 64;
+    return l;
+}
 
 struct UArgs {
     const __nv_bfloat16 *q, *k, *v, *la_f, *la_b;
     __nv_bfloat16* out;
-    int L;
+    int L, rows;
     int* dev_status;
 };
+
+// Packed bf16 values of one 32-column block of P for this thread's row.  REL < 0: the block lies left
+// of the diagonal block (forward scores only), REL > 0: right of it (backward only), REL == 0: the
+// diagonal block, forward part masked to s <= t, backward part to s >= t, summed in fp32.
+template <int REL>
+__device__ __forceinline__ void combine_block(uint32_t fwd_addr, uint32_t bwd_addr, int lane, uint32_t (&pk)[16]) {
+    if (REL != 0) {
+        uint32_t r[32];
+        tmem_ld32(REL < 0 ? fwd_addr : bwd_addr, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(as_f(r[2 * e]), as_f(r[2 * e + 1]));
+    } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t f[16], b[16];
+            tmem_ld16(fwd_addr + 16 * h, f);
+            tmem_ld16(bwd_addr + 16 * h, b);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int s0 = 16 * h + 2 * e, s1 = s0 + 1;
+                const float lo = (s0 <= lane ? as_f(f[2 * e]) : 0.f) + (s0 >= lane ? as_f(b[2 * e]) : 0.f);
+                const float hi = (s1 <= lane ? as_f(f[2 * e + 1]) : 0.f) + (s1 >= lane ? as_f(b[2 * e + 1]) : 0.f);
+                pk[8 * h + e] = pack_bf16(lo, hi);
+            }
+        }
+    }
+}
+__device__ __forceinline__ void combine_any(int cb, int wq, bool valid, uint32_t fwd_addr, uint32_t bwd_addr, int lane,
+                                            uint32_t (&pk)[16]) {
+    if (!valid) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) pk[e] = 0u;
+    } else if (cb < wq) {
+        combine_block<-1>(fwd_addr, bwd_addr, lane, pk);
+    } else if (cb == wq) {
+        combine_block<0>(fwd_addr, bwd_addr, lane, pk);
+    } else {
+        combine_block<1>(fwd_addr, bwd_addr, lane, pk);
+    }
+}
 
 template <int DK, int DV>
 __global__ void __launch_bounds__(kThreads, 2)
 bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const UArgs args) {
-    static_assert((DK == 24 || DK == 32) && (DV == 48 || DV == 64), "unsupported head size");
+    static_assert((DK == 16 || DK == 24 || DK == 32) && (DV == 32 || DV == 48 || DV == 64), "unsupported head size");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* bp = smem_raw + (base - smem_u32(smem_raw));
+    const ULayout lay = make_layout(args.rows);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int c = warp >> 2, wq = warp & 3;            // chunk and row quadrant of this warp
     const int unit = blockIdx.x, L = args.L;
-    const int nb = (L + kBlk - 1) / kBlk, nc = (L + kChunk - 1) / kChunk;
-    const uint32_t bar_tma = base + USmem::misc, bar_mma = bar_tma + 8, slot = bar_tma + 16;
-    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + USmem::misc + 16);
-    volatile int* slow_flag = reinterpret_cast<volatile int*>(bp + USmem::misc + 20);
-    float* tot = reinterpret_cast<float*>(bp + USmem::tot);
+    const int nc = (L + kChunk - 1) / kChunk;
+    const int row = c * kChunk + wq * 32 + lane;       // token owned by this thread
+    const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
+    const bool row_live = row < L;
+    const int ks0 = (min(L, kChunk) + 15) >> 4;        // 16-token K steps of chunk 0 ...
+    const int ks1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;   // ... and chunk 1
+    const uint32_t bar_tma = base + lay.misc, bar_mma = bar_tma + 8, slot = bar_tma + 16;
+    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 16);
+    volatile int* slow_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 20);
+    float* dec = reinterpret_cast<float*>(bp + lay.dec);
     uint32_t mma_phase = 0;
     bool timed_out = false;
 
@@ -139,282 +216,308 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(kTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
+    // 0/1 tiles, K-major without swizzle: 8-row groups of 256 bytes, each two 8x8 core matrices (K 0..7, K 8..15).
+    if (tid < (int)kZRows) {
+        uint32_t f[8], b[8];
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            uint32_t wf = 0, wb = 0;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int kk = 2 * p + h, u = tid - 112;
+                const bool one_f = tid >= 128 || (tid >= 112 && kk <= u);
+                const bool one_b = tid < 112 || (tid < 128 && kk >= u);
+                wf |= (one_f ? 0x3F80u : 0u) << (16 * h);
+                wb |= (one_b ? 0x3F80u : 0u) << (16 * h);
+            }
+            f[p] = wf;
+            b[p] = wb;
+        }
+        const uint32_t off = (uint32_t)(tid >> 3) * 256 + (uint32_t)(tid & 7) * 16;
+        *reinterpret_cast<uint4*>(bp + lay.zf + off) = make_uint4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<uint4*>(bp + lay.zf + off + 128) = make_uint4(f[4], f[5], f[6], f[7]);
+        *reinterpret_cast<uint4*>(bp + lay.zb + off) = make_uint4(b[0], b[1], b[2], b[3]);
+        *reinterpret_cast<uint4*>(bp + lay.zb + off + 128) = make_uint4(b[4], b[5], b[6], b[7]);
+    }
+    fence_async_smem();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *slot_p;
+    const uint32_t rc = tmem + (uint32_t)c * 128 + ((uint32_t)(wq * 32) << 16);   // this thread's lane, this chunk's columns
 
     if (tid == 0) {
-        mbar_expect_tx(bar_tma, kRows * (4 * 64 + 128));
-        tma_load_3d(base + USmem::a0 + 0 * USmem::tile, &tm_q, 0, 0, unit, bar_tma);
-        tma_load_3d(base + USmem::a0 + 1 * USmem::tile, &tm_k, 0, 0, unit, bar_tma);
-        tma_load_3d(base + USmem::a0 + 2 * USmem::tile, &tm_f, 0, 0, unit, bar_tma);
-        tma_load_3d(base + USmem::a0 + 3 * USmem::tile, &tm_b, 0, 0, unit, bar_tma);
-        tma_load_3d(base + USmem::v, &tm_v, 0, 0, unit, bar_tma);
+        mbar_expect_tx(bar_tma, (uint32_t)args.rows * (4 * 64 + 128));
+        tma_load_3d(base + 0 * lay.tile, &tm_q, 0, 0, unit, bar_tma);
+        tma_load_3d(base + 1 * lay.tile, &tm_k, 0, 0, unit, bar_tma);
+        tma_load_3d(base + 2 * lay.tile, &tm_f, 0, 0, unit, bar_tma);
+        tma_load_3d(base + 3 * lay.tile, &tm_b, 0, 0, unit, bar_tma);
+        tma_load_3d(base + lay.v, &tm_v, 0, 0, unit, bar_tma);
     }
     if (__syncthreads_or(mbar_wait_bounded(bar_tma, 0) ? 0 : 1)) {
         mbar_wait_bounded(bar_tma, 0);   // a second bounded chance for copies still in flight
         timed_out = true;
     }
 
-    if (!timed_out) {
-        // ---- phase 1a: per-block sums of log2(alpha), both directions ------------------------------
-        const int dir = lane >> 4, cp = lane & 15;
-        const bool active = cp < DK / 2;
-        const int chunk16 = cp >> 2, inchunk = (cp & 3) * 4;
-        const uint32_t q_t = base + USmem::a0, k_t = q_t + USmem::tile, g_t = q_t + (2 + dir) * USmem::tile;
-        const uint32_t kout_t = dir == 0 ? k_t : q_t;
-        for (int n = warp; n < nb; n += kThreads / 32) {
-            float sx = 0.f, sy = 0.f;
-            if (active) {
-#pragma unroll
-                for (int m = 0; m < 16; ++m) {
-                    const int r = dir == 0 ? m : 15 - m;
-                    const float2 gf = unpack_bf16(lds32(g_t + sw_off<64>(n * kBlk + r, chunk16) + inchunk));
-                    sx += gf.x;
-                    sy += gf.y;
-                }
-            }
-            *reinterpret_cast<float2*>(tot + (dir * 16 + n) * 32 + 2 * cp) = make_float2(sx * kLog2e, sy * kLog2e);
-        }
-        __syncthreads();
-
-        // ---- phase 1b: scaled operands, in place; exponents run from the chunk boundary ----------------
-        // Half-warp 0 walks a block downwards (forward gate, prefix sums), half-warp 1 upwards (backward
-        // gate, suffix sums); q~ replaces the lane's gate values at once, k~ replaces k (forward) or q
-        // (backward) from step 8 on, when both half-warps have read the row.
-        for (int n = warp; n < nb; n += kThreads / 32) {
-            const int first = n & ~7, last = min(first + 7, nb - 1);
-            float accx = 0.f, accy = 0.f;
-            if (dir == 0) {
-                for (int m = first; m < n; ++m) {
-                    const float2 t = *reinterpret_cast<const float2*>(tot + m * 32 + 2 * cp);
-                    accx += t.x; accy += t.y;
-                }
-            } else {
-                for (int m = last; m > n; --m) {
-                    const float2 t = *reinterpret_cast<const float2*>(tot + (16 + m) * 32 + 2 * cp);
-                    accx += t.x; accy += t.y;
-                }
-            }
-            uint32_t held[8];
-#pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                const int r = dir == 0 ? m : 15 - m;
-                const uint32_t off = sw_off<64>(n * kBlk + r, chunk16) + inchunk;
-                uint32_t kt = 0;
-                if (active) {
-                    const float2 qf = unpack_bf16(lds32(q_t + off));
-                    const float2 kf = unpack_bf16(lds32(k_t + off));
-                    const float2 gf = unpack_bf16(lds32(g_t + off));
-                    accx = fmaf(gf.x, kLog2e, accx);
-                    accy = fmaf(gf.y, kLog2e, accy);
-                    const float ex = ex2(accx), ey = ex2(accy), ix = ex2(-accx), iy = ex2(-accy);
-                    sts32(g_t + off, pack_bf16(qf.x * ex, qf.y * ey));   // q~ = q e^{b}
-                    kt = pack_bf16(kf.x * ix, kf.y * iy);                // k~ = k e^{-b}
-                }
-                if (m < 8) {
-                    held[m] = kt;
-                } else {
-                    __syncwarp();
-                    if (active) {
-                        sts32(kout_t + off, kt);
-                        const int r2 = dir == 0 ? 15 - m : m;
-                        sts32(kout_t + sw_off<64>(n * kBlk + r2, chunk16) + inchunk, held[15 - m]);
-                    }
-                }
-            }
-            if (active && fminf(accx, accy) < -kGateRange * kLog2e) *slow_flag = 1;
-        }
-        fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
+    auto wait_mma = [&]() -> bool {
+        const int bad = mbar_wait_bounded(bar_mma, mma_phase & 1) ? 0 : 1;
+        ++mma_phase;
+        const bool fail = __syncthreads_or(bad) != 0;
+        tc_fence_after();
+        return !fail;
+    };
+    // all threads have finished their TMEM / shared-memory accesses -> the issuing thread may start the next MMAs
+    auto handover = [&]() {
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-    }
+    };
 
-    const bool slow = !timed_out && *slow_flag != 0;
-    if (!timed_out && !slow) {
-        const int wq = warp & 3, half = warp >> 2;
-        const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
-        constexpr uint32_t kIdP = instr_desc(128, 128, 0, 0);
-        constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
-        constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
-        const uint32_t aT = base + USmem::a0, vT = base + USmem::v;
+    const uint32_t t_kb = base, t_kf = base + lay.tile, t_qf = base + 2 * lay.tile, t_qb = base + 3 * lay.tile;
+    const uint32_t t_v = base + lay.v;
+    bool slow = false;
 
-        // P of one direction for chunk c -> T1 (issued by one thread)
-        auto issue_p = [&](int c, int d) {
-            const uint32_t qa = aT + (2 + d) * USmem::tile + c * (kChunk * 64);
-            const uint32_t ka = aT + (d == 0 ? 1 : 0) * USmem::tile + c * (kChunk * 64);
-#pragma unroll
-            for (int kk = 0; kk < 2; ++kk)
-                umma_ss(tmem + kT1, smem_desc(qa + kk * 32, 16, 512, 4), smem_desc(ka + kk * 32, 16, 512, 4), kIdP, kk > 0);
-        };
-        auto issue_u = [&](int c, uint32_t dcol) {
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                umma_ss(tmem + dcol, smem_desc(aT + c * (kChunk * 64) + kk * 1024, USmem::tile, 512, 4),
-                        smem_desc(vT + c * (kChunk * 128) + kk * 2048, 16, 1024, 2), kIdU, kk > 0);
-        };
-        auto issue_o = [&](int c) {
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                umma_ts(tmem + kTO, tmem + kT1 + kk * 8, smem_desc(vT + c * (kChunk * 128) + kk * 2048, 16, 1024, 2), kIdO,
-                        kk > 0);
-            if (nc == 2) {
-                // inter-chunk term: chunk 1 gets the forward state of chunk 0, chunk 0 the backward state of chunk 1
-                const uint32_t qa = aT + (c == 1 ? 2 : 3) * USmem::tile + c * (kChunk * 64);
-                const uint32_t sa = base + (c == 1 ? USmem::s_fwd : USmem::s_bwd);
-#pragma unroll
-                for (int kk = 0; kk < 2; ++kk)
-                    umma_ss(tmem + kTO, smem_desc(qa + kk * 32, 16, 512, 4), smem_desc(sa + kk * 2048, 16, 1024, 2), kIdO, 1);
-            }
-        };
-        auto wait_mma = [&]() -> bool {
-            const int bad = mbar_wait_bounded(bar_mma, mma_phase & 1) ? 0 : 1;
-            ++mma_phase;
-            const bool fail = __syncthreads_or(bad) != 0;
-            tc_fence_after();
-            return !fail;
-        };
-
+    if (!timed_out) {
+        // ---- prefix / suffix sums of the log gates -> columns [0,32) / [32,64) of each chunk's TMEM block ----
         if (tid == 0) {
-            if (nc == 2) {
-                issue_u(0, kTU);
-                issue_u(1, kTO);
-            }
-            issue_p(0, 0);
-            umma_commit(bar_mma);
-        }
-
-        for (int c = 0; c < nc && !timed_out; ++c) {
-            const int rows_here = min(kChunk, L - c * kChunk);
-            const bool rows_live = wq * 32 < rows_here;   // this warp's 32 rows hold at least one token
-            uint32_t pk[2][16];
-            float dg[32];
-            if (!wait_mma()) { timed_out = true; break; }
-
-            // forward part of P: column blocks below the diagonal, and the diagonal block masked to s <= t
-            if (rows_live) {
-#pragma unroll
-                for (int bl = 0; bl < 2; ++bl) {
-                    const int cb = 2 * half + bl;
-                    if (cb < wq) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + kT1 + lane_base + cb * 32, r);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            pk[bl][e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                    } else if (cb == wq) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + kT1 + lane_base + cb * 32, r);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) dg[e] = e <= lane ? __uint_as_float(r[e]) : 0.f;
-                    }
+            constexpr uint32_t kIdS = instr_desc(128, 32, 0, 1);
+            for (int cc = 0; cc < nc; ++cc) {
+                const int ks = cc == 0 ? ks0 : ks1;
+                for (int j = 0; j < ks; ++j) {
+                    const uint32_t win = (uint32_t)(14 - 2 * j) * 256;        // window start row 112 - 16 j
+                    const uint32_t rows_off = (uint32_t)(cc * kChunk + 16 * j) * 64;
+                    umma_ss(tmem + cc * 128 + 0, smem_desc(base + lay.zf + win, 128, 256, 0),
+                            smem_desc(t_qf + rows_off, 16, 512, 4), kIdS, j > 0);
+                    umma_ss(tmem + cc * 128 + 32, smem_desc(base + lay.zb + win, 128, 256, 0),
+                            smem_desc(t_qb + rows_off, 16, 512, 4), kIdS, j > 0);
                 }
             }
-            // chunk summaries -> bf16 state tiles (first chunk only; warps 4 and 5 have no forward P work)
-            if (c == 0 && nc == 2 && (warp == 4 || warp == 5)) {
-                const bool fwd = warp == 5;   // lanes 32..63 of U hold k~>^T v, lanes 0..31 hold k~<^T v
-                const uint32_t ucol = fwd ? kTU : kTO;
-                float dsum = 0.f;
-                const int b0 = fwd ? 0 : 8, b1 = fwd ? 8 : nb;
-                for (int m = b0; m < b1; ++m) dsum += tot[((fwd ? 0 : 16) + m) * 32 + lane];
-                const float dec = ex2(dsum);   // decay of the whole chunk for key dim `lane`
-                const uint32_t st = base + (fwd ? USmem::s_fwd : USmem::s_bwd);
+            umma_commit(bar_mma);
+        }
+        if (!wait_mma()) timed_out = true;
+    }
+
+    if (!timed_out) {
+        // ---- scaled operands, in place: every thread rewrites its own row ---------------------------------
+        if (warp_live) {
+            uint32_t pf[32], pb[32];
+            tmem_ld32(rc, pf);
+            tmem_ld32(rc + 32, pb);
+            tc_wait_ld();
+            if (row_live) {
+                const int last_row = min(L, (c + 1) * kChunk) - 1;
+                if (row == last_row || row == c * kChunk) {
+                    // b is smallest at the last row of the chunk, e at its first row
+                    float mn = 0.f;
+#pragma unroll
+                    for (int d = 0; d < DK; ++d) mn = fminf(mn, row == last_row ? as_f(pf[d]) : 0.f);
+#pragma unroll
+                    for (int d = 0; d < DK; ++d) mn = fminf(mn, row == c * kChunk ? as_f(pb[d]) : 0.f);
+                    if (mn < -kGateRange) *slow_flag = 1;
+                    if (nc == 2 && row == kChunk - 1) {
+#pragma unroll
+                        for (int d = 0; d < 32; ++d) dec[d] = ex2(as_f(pf[d]) * kLog2e);
+                    }
+                    if (row == kChunk) {
+#pragma unroll
+                        for (int d = 0; d < 32; ++d) dec[32 + d] = ex2(as_f(pb[d]) * kLog2e);
+                    }
+                }
+#pragma unroll
+                for (int ch = 0; ch < DK / 8; ++ch) {
+                    const uint32_t off = sw_off<64>(row, ch);
+                    const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
+                    const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + lay.tile + off);
+                    const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w}, kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
+                    uint32_t qf[4], kf[4], qb[4], kb[4];
+#pragma unroll
+                    for (int m = 0; m < 4; ++m) {
+                        const float x0 = as_f(pf[8 * ch + 2 * m]) * kLog2e, x1 = as_f(pf[8 * ch + 2 * m + 1]) * kLog2e;
+                        const float y0 = as_f(pb[8 * ch + 2 * m]) * kLog2e, y1 = as_f(pb[8 * ch + 2 * m + 1]) * kLog2e;
+                        qf[m] = mul_bf16x2(qv[m], pack_bf16(ex2(x0), ex2(x1)));      // q~> = q e^{b}
+                        kf[m] = mul_bf16x2(kv[m], pack_bf16(ex2(-x0), ex2(-x1)));    // k~> = k e^{-b}
+                        qb[m] = mul_bf16x2(qv[m], pack_bf16(ex2(y0), ex2(y1)));      // q~< = q e^{e}
+                        kb[m] = mul_bf16x2(kv[m], pack_bf16(ex2(-y0), ex2(-y1)));    // k~< = k e^{-e}
+                    }
+                    *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+                    *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
+                    *reinterpret_cast<uint4*>(bp + 3 * lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
+                    *reinterpret_cast<uint4*>(bp + 0 * lay.tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
+                }
+            }
+        }
+        fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
+        handover();
+        slow = *slow_flag != 0;
+    }
+
+    if (!timed_out && !slow) {
+        constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
+        constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
+        uint32_t hold[32];   // packed bf16 P of this row, key columns 0..63
+
+        // ---- P, key columns [64 p, 64 p + 64): forward scores -> columns [0,64), backward -> [64,128) ----
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            const int n0 = min(ks0 * 16 - 64 * p, 64), n1 = min(ks1 * 16 - 64 * p, 64);   // key columns of this half
+            if (n0 <= 0 && n1 <= 0) break;   // block-uniform
+            if (tid == 0) {
+                for (int cc = 0; cc < nc; ++cc) {
+                    const int n = cc == 0 ? n0 : n1;
+                    if (n <= 0) continue;
+                    const uint32_t idp = instr_desc(128, n, 0, 0);
+                    const uint32_t qoff = (uint32_t)cc * (kChunk * 64), koff = (uint32_t)(cc * kChunk + 64 * p) * 64;
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {
+                        umma_ss(tmem + cc * 128 + 0, smem_desc(t_qf + qoff + kk * 32, 16, 512, 4),
+                                smem_desc(t_kf + koff + kk * 32, 16, 512, 4), idp, kk > 0);
+                        umma_ss(tmem + cc * 128 + 64, smem_desc(t_qb + qoff + kk * 32, 16, 512, 4),
+                                smem_desc(t_kb + koff + kk * 32, 16, 512, 4), idp, kk > 0);
+                    }
+                }
+                umma_commit(bar_mma);
+            }
+            if (!wait_mma()) { timed_out = true; break; }
+            if (warp_live) {
+                const int nkeys = (c == 0 ? ks0 : ks1) * 16;
+                uint32_t pk[16];
+                combine_any(2 * p, wq, 64 * p < nkeys, rc, rc + 64, lane, pk);
+                if (p == 0) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) hold[e] = pk[e];
+                } else {
+                    // key block 2 has been read: columns [0,32) are dead and take the packed first half
+                    uint32_t h0[16], h1[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) { h0[e] = hold[e]; h1[e] = hold[16 + e]; }
+                    tmem_st16(rc, h0);
+                    tmem_st16(rc + 16, h1);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) hold[e] = pk[e];
+                }
+                combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, pk);
+                if (p == 0) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) hold[16 + e] = pk[e];
+                } else {
+                    uint32_t h0[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) h0[e] = hold[e];
+                    tmem_st16(rc + 32, h0);
+                    tmem_st16(rc + 48, pk);
+                }
+            }
+            if (p == 0 && ks0 <= 4 && ks1 <= 4 && warp_live) {   // no second half: the first is all there is
+                uint32_t h0[16], h1[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) { h0[e] = hold[e]; h1[e] = hold[16 + e]; }
+                tmem_st16(rc, h0);
+                tmem_st16(rc + 16, h1);
+            }
+            tc_wait_st();
+            handover();
+        }
+
+        // ---- chunk summaries -> bf16 state tiles (two chunks only) -----------------------------------------
+        if (!timed_out && nc == 2) {
+            if (tid == 0) {
+                for (int cc = 0; cc < 2; ++cc) {
+                    const int ks = cc == 0 ? ks0 : ks1;
+                    for (int kk = 0; kk < ks; ++kk)
+                        umma_ss(tmem + cc * 128 + 64, smem_desc(t_kb + (uint32_t)cc * (kChunk * 64) + kk * 1024, lay.tile, 512, 4),
+                                smem_desc(t_v + (uint32_t)cc * (kChunk * 128) + kk * 2048, 16, 1024, 2), kIdU, kk > 0);
+                }
+                umma_commit(bar_mma);
+            }
+            if (!wait_mma()) timed_out = true;
+            if (!timed_out && (warp == 1 || warp == 4)) {
+                // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
+                // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
+                const float d = dec[(warp == 1 ? 0 : 32) + lane];
+                const uint32_t st = base + (warp == 1 ? lay.s_fwd : lay.s_bwd);
 #pragma unroll
                 for (int hb = 0; hb < 2; ++hb) {
                     uint32_t r[32];
-                    tmem_ld32(tmem + ucol + lane_base + hb * 32, r);
+                    tmem_ld32(rc + 64 + hb * 32, r);
                     tc_wait_ld();
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
                         uint32_t o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            o[e] = pack_bf16(__uint_as_float(r[ch * 8 + 2 * e]) * dec, __uint_as_float(r[ch * 8 + 2 * e + 1]) * dec);
-                        sts128(st + sw_off<128>(lane, hb * 4 + ch), o[0], o[1], o[2], o[3]);
+                        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(as_f(r[ch * 8 + 2 * e]) * d, as_f(r[ch * 8 + 2 * e + 1]) * d);
+                        *reinterpret_cast<uint4*>(bp + (st - base) + sw_off<128>(lane, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
                 fence_async_smem();
             }
-            tc_fence_before();
-            __syncthreads();
-            tc_fence_after();
+            handover();
+        }
+
+        // ---- out = (P v + q~ S_in) / 2 ------------------------------------------------------------------------
+        if (!timed_out) {
             if (tid == 0) {
-                issue_p(c, 1);
+                for (int cc = 0; cc < nc; ++cc) {
+                    const int ks = cc == 0 ? ks0 : ks1;
+                    uint32_t acc = 0;
+                    if (nc == 2) {
+                        // chunk 1 receives the forward state of chunk 0, chunk 0 the backward state of chunk 1
+                        const uint32_t qa = (cc == 1 ? t_qf : t_qb) + (uint32_t)cc * (kChunk * 64);
+                        const uint32_t sa = base + (cc == 1 ? lay.s_fwd : lay.s_bwd);
+#pragma unroll
+                        for (int kk = 0; kk < 2; ++kk) {
+                            umma_ss(tmem + cc * 128 + 64, smem_desc(qa + kk * 32, 16, 512, 4), smem_desc(sa + kk * 2048, 16, 1024, 2),
+                                    kIdO, acc);
+                            acc = 1;
+                        }
+                    }
+                    for (int kk = 0; kk < ks; ++kk) {
+                        umma_ts(tmem + cc * 128 + 64, tmem + cc * 128 + kk * 8,
+                                smem_desc(t_v + (uint32_t)cc * (kChunk * 128) + kk * 2048, 16, 1024, 2), kIdO, acc);
+                        acc = 1;
+                    }
+                }
                 umma_commit(bar_mma);
             }
-            if (!wait_mma()) { timed_out = true; break; }
-
-            // backward part of P, combine, pack, and put bf16 P where the P v MMA reads it
-            if (rows_live) {
+            if (!wait_mma()) timed_out = true;
+        }
+        if (!timed_out) {
+            // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
+            if (warp_live) {
 #pragma unroll
-                for (int bl = 0; bl < 2; ++bl) {
-                    const int cb = 2 * half + bl;
-                    if (cb > wq) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + kT1 + lane_base + cb * 32, r);
-                        tc_wait_ld();
+                for (int hb = 0; hb < DV / 32; ++hb) {
+                    uint32_t r[32];
+                    tmem_ld32(rc + 64 + hb * 32, r);
+                    tc_wait_ld();
+                    if (row_live) {
 #pragma unroll
-                        for (int e = 0; e < 16; ++e)
-                            pk[bl][e] = pack_bf16(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1]));
-                    } else if (cb == wq) {
-                        uint32_t r[32];
-                        tmem_ld32(tmem + kT1 + lane_base + cb * 32, r);
-                        tc_wait_ld();
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t o[4];
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const float lo = (2 * e >= lane ? __uint_as_float(r[2 * e]) : 0.f) + dg[2 * e];
-                            const float hi = (2 * e + 1 >= lane ? __uint_as_float(r[2 * e + 1]) : 0.f) + dg[2 * e + 1];
-                            pk[bl][e] = pack_bf16(lo, hi);
+                            for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
+                            *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                }
+                if (DV == 48) {
+                    uint32_t r[16];
+                    tmem_ld16(rc + 64 + 32, r);
+                    tc_wait_ld();
+                    if (row_live) {
+#pragma unroll
+                        for (int ch = 0; ch < 2; ++ch) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
+                            *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                         }
                     }
                 }
             }
-            named_bar(1 + wq, 64);   // both warps of this row quadrant have finished reading fp32 P
-            if (rows_live) {
-#pragma unroll
-                for (int bl = 0; bl < 2; ++bl) tmem_st16(tmem + kT1 + lane_base + (2 * half + bl) * 16, pk[bl]);
-                tc_wait_st();
-            }
+            fence_async_smem();
             tc_fence_before();
             __syncthreads();
-            tc_fence_after();
             if (tid == 0) {
-                issue_o(c);
-                umma_commit(bar_mma);
-            }
-            if (!wait_mma()) { timed_out = true; break; }
-            if (tid == 0 && c + 1 < nc) {
-                issue_p(c + 1, 0);   // next chunk's forward P runs while this chunk's output is written out
-                umma_commit(bar_mma);
-            }
-
-            // epilogue: out = O / 2, bf16, into the dead v tile of this chunk (same swizzle as the TMA store expects)
-            if (rows_live) {
-                uint32_t r[32];
-                tmem_ld32(tmem + kTO + lane_base + half * 32, r);
-                tc_wait_ld();
-                const int row = c * kChunk + wq * 32 + lane;
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t o[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        o[e] = pack_bf16(0.5f * __uint_as_float(r[ch * 8 + 2 * e]), 0.5f * __uint_as_float(r[ch * 8 + 2 * e + 1]));
-                    sts128(vT + sw_off<128>(row, half * 4 + ch), o[0], o[1], o[2], o[3]);
-                }
-            }
-            tc_fence_before();   // the next chunk's O MMA overwrites the accumulator only after these loads
-        }
-
-        if (!timed_out) {
-            fence_async_smem();
-            __syncthreads();
-            if (tid == 0) {
-                tma_store_3d(&tm_o, 0, 0, unit, vT);   // rows >= L and columns >= dv are clipped
+                tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             }
@@ -441,16 +544,19 @@ template <int DK, int DV>
 cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                           const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units, int L,
                           cudaStream_t stream) {
+    const int rows = (L + 15) / 16 * 16;
     CUtensorMap tq, tk, tf, tb, tv, to;
-    if (!make_map(&tq, q, units, L, DK, 32, kRows) || !make_map(&tk, k, units, L, DK, 32, kRows) ||
-        !make_map(&tf, la_f, units, L, DK, 32, kRows) || !make_map(&tb, la_b, units, L, DK, 32, kRows) ||
-        !make_map(&tv, v, units, L, DV, 64, kRows) || !make_map(&to, out, units, L, DV, 64, kRows))
+    if (!make_map(&tq, q, units, L, DK, 32, rows) || !make_map(&tk, k, units, L, DK, 32, rows) ||
+        !make_map(&tf, la_f, units, L, DK, 32, rows) || !make_map(&tb, la_b, units, L, DK, 32, rows) ||
+        !make_map(&tv, v, units, L, DV, 64, rows) || !make_map(&to, out, units, L, DV, 64, rows))
         return cudaErrorInvalidValue;
     UArgs a{};
-    a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L;
+    a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows;
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
-    size_t smem = USmem::total + 1024;
+    // The MMAs of chunk 1 read 128 rows of the operand tiles from row 128 on, i.e. up to (256 - rows) * 64
+    // bytes past the last q-type tile: that lands in the v tile, inside the allocation.
+    size_t smem = make_layout(rows).total + 1024;   // slack for the manual 1 KB alignment
     const size_t rec = (size_t)rec_plan(kThreads, DK, DV).smem_floats * 4 + 1024;
     if (smem < rec) smem = rec;
     cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -462,14 +568,18 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
 
 }  // namespace
 
-bool umma_supported(int dk, int dv, int L) { return (dk == 24 || dk == 32) && (dv == 48 || dv == 64) && L <= kRows; }
+bool umma_supported(int dk, int dv, int L) {
+    return (dk == 16 || dk == 24 || dk == 32) && (dv == 32 || dv == 48 || dv == 64) && L <= kMaxRows;
+}
 
 cudaError_t launch_bigla_umma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                               const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
                               int L, int dk, int dv, cudaStream_t stream) {
 #define VIG_CASE(DK_, DV_) \
     if (dk == DK_ && dv == DV_) return launch_umma_t<DK_, DV_>(q, k, v, la_f, la_b, out, units, L, stream);
-    VIG_CASE(24, 48) VIG_CASE(24, 64) VIG_CASE(32, 48) VIG_CASE(32, 64)
+    VIG_CASE(16, 32) VIG_CASE(16, 48) VIG_CASE(16, 64)
+    VIG_CASE(24, 32) VIG_CASE(24, 48) VIG_CASE(24, 64)
+    VIG_CASE(32, 32) VIG_CASE(32, 48) VIG_CASE(32, 64)
 #undef VIG_CASE
     return cudaErrorNotSupported;
 }
