@@ -46,12 +46,6 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Shared-memory matrix descriptor (start address, leading / stride byte offsets in 16-byte units,
-// descriptor version 1, swizzle mode in bits 61..63: 0 = none, 2 = 128B, 4 = 64B).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swizzle) {
-    return (uint64_t)((addr >> 4) & 0x3FFF) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) | ((uint64_t)1 << 46) | ((uint64_t)swizzle << 61);
-}
 // Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, majors, N >> 3, M >> 4.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
@@ -113,7 +107,7 @@ struct ULayout {
     uint32_t s_fwd;    // bf16 state entering chunk 1 from the left  [32][64] (128B swizzle)
     uint32_t s_bwd;    // bf16 state entering chunk 0 from the right
     uint32_t dec;      // [2][32] fp32 chunk decay factors e^{b_last} (fwd, chunk 0), e^{e_first} (bwd, chunk 1)
-    uint32_t misc;     // mbarriers, TMEM slot, flag
+    uint32_t misc;     // five mbarriers, TMEM slot, flags
     uint32_t total;
 };
 __host__ __device__ inline ULayout make_layout(int rows) {
@@ -126,7 +120,7 @@ __host__ __device__ inline ULayout make_layout(int rows) {
     l.s_bwd = l.s_fwd + 32 * 128;
     l.dec = l.s_bwd + 32 * 128;
     l.misc = l.dec + 2 * 32 * 4;
-    l.total = l.misc + 64;
+    l.total = l.misc + 128;
     return l;
 }
 
@@ -134,6 +128,7 @@ struct UArgs {
     const __nv_bfloat16 *q, *k, *v, *la_f, *la_b;
     __nv_bfloat16* out;
     int L, rows;
+    long long units;
     int* dev_status;
 };
 
@@ -179,6 +174,31 @@ __device__ __forceinline__ void combine_any(int cb, int wq, bool valid, uint32_t
     }
 }
 
+// Shared-memory matrix descriptor, in halves.  Low word: start address and leading-dimension byte
+// offset, both in 16-byte units (bits 0..13 and 16..29), so stepping an operand through shared memory is
+// one 32-bit add.  High word: stride-dimension byte offset in 16-byte units (bits 32..45), descriptor
+// version 1 (bit 46), swizzle mode in bits 61..63 (0 = none, 2 = 128B, 4 = 64B).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+    return ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes, uint32_t swizzle) {
+    return (sbo_bytes >> 4) | (1u << 14) | (swizzle << 29);
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
+
+constexpr uint32_t kHiK64 = desc_hi(512, 4);     // K-major or MN-major tile with 64-byte rows, 64B swizzle
+constexpr uint32_t kHiV128 = desc_hi(1024, 2);   // MN-major tile with 128-byte rows, 128B swizzle
+constexpr uint32_t kHiZ = desc_hi(256, 0);       // 0/1 tiles, no swizzle
+
+// 1 / x for a normal, positive x without the special-function unit: a bit-level first guess (within 5.1 %)
+// and two Newton steps (relative error below 1e-5).
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r = __uint_as_float(0x7EF311C7u - __float_as_uint(x));
+    r = r * fmaf(-x, r, 2.0f);
+    r = r * fmaf(-x, r, 2.0f);
+    return r;
+}
+
 template <int DK, int DV>
 __global__ void __launch_bounds__(kThreads, 2)
 bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -192,26 +212,52 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = warp >> 2, wq = warp & 3;            // chunk and row quadrant of this warp
-    const int unit = blockIdx.x, L = args.L;
+    const int L = args.L;
     const int nc = (L + kChunk - 1) / kChunk;
     const int row = c * kChunk + wq * 32 + lane;       // token owned by this thread
     const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
     const bool row_live = row < L;
-    const int ks0 = (min(L, kChunk) + 15) >> 4;        // 16-token K steps of chunk 0 ...
-    const int ks1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;   // ... and chunk 1
-    const uint32_t bar_tma = base + lay.misc, bar_mma = bar_tma + 8, slot = bar_tma + 16;
-    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 16);
-    volatile int* slow_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 20);
+    const bool chunk_on = c < nc;
+    const bool issuer = tid == c * kChunk;             // one thread per chunk issues that chunk's MMAs
+    const int ks = chunk_on ? (min(L - c * kChunk, kChunk) + 15) >> 4 : 0;   // 16-token K steps of this chunk
+    const int nkeys = ks * 16;
+    // mbarriers: log-gate tiles landed, q and k landed, v landed, MMA batches of chunk 0 / chunk 1
+    const uint32_t bar_g = base + lay.misc, bar_qk = bar_g + 8, bar_v = bar_g + 16, bar_mma = bar_g + 24 + 8 * c;
+    const uint32_t slot = bar_g + 40;
+    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 40);
+    volatile int* time_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 44);
+    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 48);   // [4]: (chunk, first / last row) range checks
     float* dec = reinterpret_cast<float*>(bp + lay.dec);
     uint32_t mma_phase = 0;
-    bool timed_out = false;
+
+    const uint32_t t_kb = base, t_kf = base + lay.tile, t_qf = base + 2 * lay.tile, t_qb = base + 3 * lay.tile;
+    const uint32_t t_v = base + lay.v;
+    const uint32_t g_bytes = (uint32_t)args.rows * 128, v_bytes = (uint32_t)args.rows * 128;
+    auto load_gates_qk = [&](int unit) {
+        mbar_expect_tx(bar_g, g_bytes);
+        tma_load_3d(t_qf, &tm_f, 0, 0, unit, bar_g);
+        tma_load_3d(t_qb, &tm_b, 0, 0, unit, bar_g);
+        mbar_expect_tx(bar_qk, g_bytes);
+        tma_load_3d(t_kb, &tm_q, 0, 0, unit, bar_qk);
+        tma_load_3d(t_kf, &tm_k, 0, 0, unit, bar_qk);
+    };
+    auto load_v = [&](int unit) {
+        mbar_expect_tx(bar_v, v_bytes);
+        tma_load_3d(t_v, &tm_v, 0, 0, unit, bar_v);
+    };
 
     if (tid == 0) {
-        mbar_init(bar_tma, 1);
-        mbar_init(bar_mma, 1);
-        *slow_flag = 0;
+#pragma unroll
+        for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
+        *time_flag = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) slow_slot[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // the first loads go out at once: the rest of the set-up overlaps their latency
+        load_gates_qk(blockIdx.x);
+        load_v(blockIdx.x);
     }
+    __syncwarp();
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(kTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
@@ -244,243 +290,243 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *slot_p;
-    const uint32_t rc = tmem + (uint32_t)c * 128 + ((uint32_t)(wq * 32) << 16);   // this thread's lane, this chunk's columns
+    const uint32_t tc = tmem + (uint32_t)c * 128;                   // this chunk's 128 TMEM columns
+    const uint32_t rc = tc + ((uint32_t)(wq * 32) << 16);           // ... at this thread's lane
 
-    if (tid == 0) {
-        mbar_expect_tx(bar_tma, (uint32_t)args.rows * (4 * 64 + 128));
-        tma_load_3d(base + 0 * lay.tile, &tm_q, 0, 0, unit, bar_tma);
-        tma_load_3d(base + 1 * lay.tile, &tm_k, 0, 0, unit, bar_tma);
-        tma_load_3d(base + 2 * lay.tile, &tm_f, 0, 0, unit, bar_tma);
-        tma_load_3d(base + 3 * lay.tile, &tm_b, 0, 0, unit, bar_tma);
-        tma_load_3d(base + lay.v, &tm_v, 0, 0, unit, bar_tma);
-    }
-    if (__syncthreads_or(mbar_wait_bounded(bar_tma, 0) ? 0 : 1)) {
-        mbar_wait_bounded(bar_tma, 0);   // a second bounded chance for copies still in flight
-        timed_out = true;
-    }
-
-    auto wait_mma = [&]() -> bool {
-        const int bad = mbar_wait_bounded(bar_mma, mma_phase & 1) ? 0 : 1;
+    // A bounded wait that expires raises the flag and lets the block finish the unit on whatever it has:
+    // every later wait is bounded too, nothing more is stored, and the host sees the device status word.
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
+        if (!mbar_wait_bounded(bar, parity)) *time_flag = 1;
+    };
+    auto wait_mma = [&]() {
+        wait_bar(bar_mma, mma_phase & 1);
         ++mma_phase;
-        const bool fail = __syncthreads_or(bad) != 0;
         tc_fence_after();
-        return !fail;
     };
-    // all threads have finished their TMEM / shared-memory accesses -> the issuing thread may start the next MMAs
-    auto handover = [&]() {
+    // the threads of this chunk have finished their TMEM / shared-memory accesses -> its issuer may go on
+    auto chunk_handover = [&]() {
         tc_fence_before();
-        __syncthreads();
+        named_bar(1 + c, kChunk);
         tc_fence_after();
     };
+    const uint32_t row0_64 = (uint32_t)c * (kChunk * 64) >> 4, row0_128 = (uint32_t)c * (kChunk * 128) >> 4;   // in descriptor units
 
-    const uint32_t t_kb = base, t_kf = base + lay.tile, t_qf = base + 2 * lay.tile, t_qb = base + 3 * lay.tile;
-    const uint32_t t_v = base + lay.v;
-    bool slow = false;
-
-    if (!timed_out) {
-        // ---- prefix / suffix sums of the log gates -> columns [0,32) / [32,64) of each chunk's TMEM block ----
-        if (tid == 0) {
-            constexpr uint32_t kIdS = instr_desc(128, 32, 0, 1);
-            for (int cc = 0; cc < nc; ++cc) {
-                const int ks = cc == 0 ? ks0 : ks1;
-                for (int j = 0; j < ks; ++j) {
-                    const uint32_t win = (uint32_t)(14 - 2 * j) * 256;        // window start row 112 - 16 j
-                    const uint32_t rows_off = (uint32_t)(cc * kChunk + 16 * j) * 64;
-                    umma_ss(tmem + cc * 128 + 0, smem_desc(base + lay.zf + win, 128, 256, 0),
-                            smem_desc(t_qf + rows_off, 16, 512, 4), kIdS, j > 0);
-                    umma_ss(tmem + cc * 128 + 32, smem_desc(base + lay.zb + win, 128, 256, 0),
-                            smem_desc(t_qb + rows_off, 16, 512, 4), kIdS, j > 0);
-                }
-            }
-            umma_commit(bar_mma);
+    // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
+    uint32_t it = 0;
+    bool v_load_pending = false;   // thread 0: the v tile of the current unit has not been requested yet
+    for (long long unit_ll = blockIdx.x; unit_ll < args.units; unit_ll += gridDim.x, ++it) {
+        const int unit = (int)unit_ll;
+        const uint32_t par = it & 1;
+        const bool has_next = unit_ll + gridDim.x < args.units;
+        if (tid == 32 && has_next) {
+            // pull the tiles of this block's next unit into L2
+            const int pu = unit + (int)gridDim.x;
+            tma_prefetch_3d(&tm_f, 0, 0, pu);
+            tma_prefetch_3d(&tm_b, 0, 0, pu);
+            tma_prefetch_3d(&tm_q, 0, 0, pu);
+            tma_prefetch_3d(&tm_k, 0, 0, pu);
+            tma_prefetch_3d(&tm_v, 0, 0, pu);
         }
-        if (!wait_mma()) timed_out = true;
-    }
 
-    if (!timed_out) {
-        // ---- scaled operands, in place: every thread rewrites its own row ---------------------------------
-        if (warp_live) {
-            uint32_t pf[32], pb[32];
-            tmem_ld32(rc, pf);
-            tmem_ld32(rc + 32, pb);
-            tc_wait_ld();
-            if (row_live) {
-                const int last_row = min(L, (c + 1) * kChunk) - 1;
-                if (row == last_row || row == c * kChunk) {
-                    // b is smallest at the last row of the chunk, e at its first row
-                    float mn = 0.f;
+        if (chunk_on) {
+            // ---- prefix / suffix sums of the log gates -> columns [0,32) / [32,64) of the chunk's TMEM block ----
+            wait_bar(bar_g, par);
+            if (issuer) {
+                constexpr uint32_t kIdS = instr_desc(128, 32, 0, 1);
+                const uint32_t zf = desc_lo(base + lay.zf, 128), zb = desc_lo(base + lay.zb, 128);
+                const uint32_t gf = desc_lo(t_qf, 16) + row0_64, gb = desc_lo(t_qb, 16) + row0_64;
 #pragma unroll
-                    for (int d = 0; d < DK; ++d) mn = fminf(mn, row == last_row ? as_f(pf[d]) : 0.f);
-#pragma unroll
-                    for (int d = 0; d < DK; ++d) mn = fminf(mn, row == c * kChunk ? as_f(pb[d]) : 0.f);
-                    if (mn < -kGateRange) *slow_flag = 1;
-                    if (nc == 2 && row == kChunk - 1) {
-#pragma unroll
-                        for (int d = 0; d < 32; ++d) dec[d] = ex2(as_f(pf[d]) * kLog2e);
-                    }
-                    if (row == kChunk) {
-#pragma unroll
-                        for (int d = 0; d < 32; ++d) dec[32 + d] = ex2(as_f(pb[d]) * kLog2e);
-                    }
-                }
-#pragma unroll
-                for (int ch = 0; ch < DK / 8; ++ch) {
-                    const uint32_t off = sw_off<64>(row, ch);
-                    const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
-                    const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + lay.tile + off);
-                    const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w}, kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
-                    uint32_t qf[4], kf[4], qb[4], kb[4];
-#pragma unroll
-                    for (int m = 0; m < 4; ++m) {
-                        const float x0 = as_f(pf[8 * ch + 2 * m]) * kLog2e, x1 = as_f(pf[8 * ch + 2 * m + 1]) * kLog2e;
-                        const float y0 = as_f(pb[8 * ch + 2 * m]) * kLog2e, y1 = as_f(pb[8 * ch + 2 * m + 1]) * kLog2e;
-                        qf[m] = mul_bf16x2(qv[m], pack_bf16(ex2(x0), ex2(x1)));      // q~> = q e^{b}
-                        kf[m] = mul_bf16x2(kv[m], pack_bf16(ex2(-x0), ex2(-x1)));    // k~> = k e^{-b}
-                        qb[m] = mul_bf16x2(qv[m], pack_bf16(ex2(y0), ex2(y1)));      // q~< = q e^{e}
-                        kb[m] = mul_bf16x2(kv[m], pack_bf16(ex2(-y0), ex2(-y1)));    // k~< = k e^{-e}
-                    }
-                    *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
-                    *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
-                    *reinterpret_cast<uint4*>(bp + 3 * lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
-                    *reinterpret_cast<uint4*>(bp + 0 * lay.tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
-                }
-            }
-        }
-        fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
-        handover();
-        slow = *slow_flag != 0;
-    }
-
-    if (!timed_out && !slow) {
-        constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
-        constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
-        uint32_t hold[32];   // packed bf16 P of this row, key columns 0..63
-
-        // ---- P, key columns [64 p, 64 p + 64): forward scores -> columns [0,64), backward -> [64,128) ----
-#pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            const int n0 = min(ks0 * 16 - 64 * p, 64), n1 = min(ks1 * 16 - 64 * p, 64);   // key columns of this half
-            if (n0 <= 0 && n1 <= 0) break;   // block-uniform
-            if (tid == 0) {
-                for (int cc = 0; cc < nc; ++cc) {
-                    const int n = cc == 0 ? n0 : n1;
-                    if (n <= 0) continue;
-                    const uint32_t idp = instr_desc(128, n, 0, 0);
-                    const uint32_t qoff = (uint32_t)cc * (kChunk * 64), koff = (uint32_t)(cc * kChunk + 64 * p) * 64;
-#pragma unroll
-                    for (int kk = 0; kk < 2; ++kk) {
-                        umma_ss(tmem + cc * 128 + 0, smem_desc(t_qf + qoff + kk * 32, 16, 512, 4),
-                                smem_desc(t_kf + koff + kk * 32, 16, 512, 4), idp, kk > 0);
-                        umma_ss(tmem + cc * 128 + 64, smem_desc(t_qb + qoff + kk * 32, 16, 512, 4),
-                                smem_desc(t_kb + koff + kk * 32, 16, 512, 4), idp, kk > 0);
+                for (int j = 0; j < 8; ++j) {
+                    if (j < ks) {
+                        const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+                        umma_ss(tc + 0, desc64(zf + win, kHiZ), desc64(gf + j * 64, kHiK64), kIdS, j > 0);
+                        umma_ss(tc + 32, desc64(zb + win, kHiZ), desc64(gb + j * 64, kHiK64), kIdS, j > 0);
                     }
                 }
                 umma_commit(bar_mma);
             }
-            if (!wait_mma()) { timed_out = true; break; }
+            wait_mma();
+            wait_bar(bar_qk, par);
+
+            // ---- scaled operands, in place: every thread rewrites its own row ---------------------------------
             if (warp_live) {
-                const int nkeys = (c == 0 ? ks0 : ks1) * 16;
-                uint32_t pk[16];
-                combine_any(2 * p, wq, 64 * p < nkeys, rc, rc + 64, lane, pk);
-                if (p == 0) {
+                uint32_t pf[32], pb[32];
+                tmem_ld32(rc, pf);
+                tmem_ld32(rc + 32, pb);
+                tc_wait_ld();
+                if (row_live) {
+                    const int last_row = min(L, (c + 1) * kChunk) - 1;
+                    if (row == last_row || row == c * kChunk) {
+                        // b is smallest at the last row of the chunk, e at its first row
+                        float mf = 0.f, mb = 0.f;
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) hold[e] = pk[e];
-                } else {
-                    // key block 2 has been read: columns [0,32) are dead and take the packed first half
-                    uint32_t h0[16], h1[16];
+                        for (int d = 0; d < DK; ++d) { mf = fminf(mf, as_f(pf[d])); mb = fminf(mb, as_f(pb[d])); }
+                        if (row == last_row) slow_slot[2 * c + 1] = mf < -kGateRange ? 1 : 0;
+                        if (row == c * kChunk) slow_slot[2 * c] = mb < -kGateRange ? 1 : 0;
+                        if (nc == 2 && row == kChunk - 1) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) { h0[e] = hold[e]; h1[e] = hold[16 + e]; }
-                    tmem_st16(rc, h0);
-                    tmem_st16(rc + 16, h1);
+                            for (int d = 0; d < 32; ++d) dec[d] = ex2(as_f(pf[d]) * kLog2e);
+                        }
+                        if (row == kChunk) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) hold[e] = pk[e];
-                }
-                combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, pk);
-                if (p == 0) {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) hold[16 + e] = pk[e];
-                } else {
-                    uint32_t h0[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) h0[e] = hold[e];
-                    tmem_st16(rc + 32, h0);
-                    tmem_st16(rc + 48, pk);
-                }
-            }
-            if (p == 0 && ks0 <= 4 && ks1 <= 4 && warp_live) {   // no second half: the first is all there is
-                uint32_t h0[16], h1[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) { h0[e] = hold[e]; h1[e] = hold[16 + e]; }
-                tmem_st16(rc, h0);
-                tmem_st16(rc + 16, h1);
-            }
-            tc_wait_st();
-            handover();
-        }
-
-        // ---- chunk summaries -> bf16 state tiles (two chunks only) -----------------------------------------
-        if (!timed_out && nc == 2) {
-            if (tid == 0) {
-                for (int cc = 0; cc < 2; ++cc) {
-                    const int ks = cc == 0 ? ks0 : ks1;
-                    for (int kk = 0; kk < ks; ++kk)
-                        umma_ss(tmem + cc * 128 + 64, smem_desc(t_kb + (uint32_t)cc * (kChunk * 64) + kk * 1024, lay.tile, 512, 4),
-                                smem_desc(t_v + (uint32_t)cc * (kChunk * 128) + kk * 2048, 16, 1024, 2), kIdU, kk > 0);
-                }
-                umma_commit(bar_mma);
-            }
-            if (!wait_mma()) timed_out = true;
-            if (!timed_out && (warp == 1 || warp == 4)) {
-                // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
-                // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
-                const float d = dec[(warp == 1 ? 0 : 32) + lane];
-                const uint32_t st = base + (warp == 1 ? lay.s_fwd : lay.s_bwd);
-#pragma unroll
-                for (int hb = 0; hb < 2; ++hb) {
-                    uint32_t r[32];
-                    tmem_ld32(rc + 64 + hb * 32, r);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint32_t o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(as_f(r[ch * 8 + 2 * e]) * d, as_f(r[ch * 8 + 2 * e + 1]) * d);
-                        *reinterpret_cast<uint4*>(bp + (st - base) + sw_off<128>(lane, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                }
-                fence_async_smem();
-            }
-            handover();
-        }
-
-        // ---- out = (P v + q~ S_in) / 2 ------------------------------------------------------------------------
-        if (!timed_out) {
-            if (tid == 0) {
-                for (int cc = 0; cc < nc; ++cc) {
-                    const int ks = cc == 0 ? ks0 : ks1;
-                    uint32_t acc = 0;
-                    if (nc == 2) {
-                        // chunk 1 receives the forward state of chunk 0, chunk 0 the backward state of chunk 1
-                        const uint32_t qa = (cc == 1 ? t_qf : t_qb) + (uint32_t)cc * (kChunk * 64);
-                        const uint32_t sa = base + (cc == 1 ? lay.s_fwd : lay.s_bwd);
-#pragma unroll
-                        for (int kk = 0; kk < 2; ++kk) {
-                            umma_ss(tmem + cc * 128 + 64, smem_desc(qa + kk * 32, 16, 512, 4), smem_desc(sa + kk * 2048, 16, 1024, 2),
-                                    kIdO, acc);
-                            acc = 1;
+                            for (int d = 0; d < 32; ++d) dec[32 + d] = ex2(as_f(pb[d]) * kLog2e);
                         }
                     }
-                    for (int kk = 0; kk < ks; ++kk) {
-                        umma_ts(tmem + cc * 128 + 64, tmem + cc * 128 + kk * 8,
-                                smem_desc(t_v + (uint32_t)cc * (kChunk * 128) + kk * 2048, 16, 1024, 2), kIdO, acc);
-                        acc = 1;
+#pragma unroll
+                    for (int ch = 0; ch < DK / 8; ++ch) {
+                        const uint32_t off = sw_off<64>(row, ch);
+                        const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
+                        const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + lay.tile + off);
+                        const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w}, kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
+                        uint32_t qf[4], kf[4], qb[4], kb[4];
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            // e^{b} on the special-function unit, e^{-b} as its reciprocal on the FMA pipe
+                            const float ex0 = ex2(as_f(pf[8 * ch + 2 * m]) * kLog2e), ex1 = ex2(as_f(pf[8 * ch + 2 * m + 1]) * kLog2e);
+                            const float ey0 = ex2(as_f(pb[8 * ch + 2 * m]) * kLog2e), ey1 = ex2(as_f(pb[8 * ch + 2 * m + 1]) * kLog2e);
+                            qf[m] = mul_bf16x2(qv[m], pack_bf16(ex0, ex1));                        // q~> = q e^{b}
+                            kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp(ex0), fast_rcp(ex1)));    // k~> = k e^{-b}
+                            qb[m] = mul_bf16x2(qv[m], pack_bf16(ey0, ey1));                        // q~< = q e^{e}
+                            kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp(ey0), fast_rcp(ey1)));    // k~< = k e^{-e}
+                        }
+                        *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+                        *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
+                        *reinterpret_cast<uint4*>(bp + 3 * lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
+                        *reinterpret_cast<uint4*>(bp + 0 * lay.tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
+                    }
+                }
+            }
+            fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
+            chunk_handover();
+            if (tid == 0 && v_load_pending) {
+                // The store of the previous unit was issued a phase ago and has read the v tile by now: this
+                // wait is short, and the tile is only needed again when the chunk summaries are formed.
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                load_v(unit);
+                v_load_pending = false;
+            }
+
+            // ---- P, key columns [64 p, 64 p + 64): forward scores -> columns [0,64), backward -> [64,128) ----
+            uint32_t hold[32];   // packed bf16 P of this row, key columns 0..63
+            const uint32_t aqf = desc_lo(t_qf, 16) + row0_64, aqb = desc_lo(t_qb, 16) + row0_64;
+            const uint32_t bkf = desc_lo(t_kf, 16) + row0_64, bkb = desc_lo(t_kb, 16) + row0_64;
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+                const int n = min(nkeys - 64 * p, 64);   // key columns of this half
+                if (n <= 0) break;
+                if (issuer) {
+                    const uint32_t idp = instr_desc(128, n, 0, 0);
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) {
+                        umma_ss(tc + 0, desc64(aqf + kk * 2, kHiK64), desc64(bkf + p * 256 + kk * 2, kHiK64), idp, kk > 0);
+                        umma_ss(tc + 64, desc64(aqb + kk * 2, kHiK64), desc64(bkb + p * 256 + kk * 2, kHiK64), idp, kk > 0);
+                    }
+                    umma_commit(bar_mma);
+                }
+                wait_mma();
+                if (warp_live) {
+                    uint32_t pk[16];
+                    combine_any(2 * p, wq, true, rc, rc + 64, lane, pk);
+                    if (p == 0) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) hold[e] = pk[e];
+                    } else {
+                        // key block 2 has been read: columns [0,32) are dead and take the packed first half
+                        uint32_t h0[16], h1[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) { h0[e] = hold[e]; h1[e] = hold[16 + e]; }
+                        tmem_st16(rc, h0);
+                        tmem_st16(rc + 16, h1);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) hold[e] = pk[e];
+                    }
+                    combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, pk);
+                    if (p == 0) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) hold[16 + e] = pk[e];
+                        if (nkeys <= 64) {   // no second half
+                            uint32_t h0[16];
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) h0[e] = hold[e];
+                            tmem_st16(rc, h0);
+                            tmem_st16(rc + 16, pk);
+                        }
+                    } else {
+                        uint32_t h0[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) h0[e] = hold[e];
+                        tmem_st16(rc + 32, h0);
+                        tmem_st16(rc + 48, pk);
+                    }
+                }
+                tc_wait_st();
+                chunk_handover();
+            }
+
+            // ---- chunk summary -> bf16 state tile for the other chunk (two chunks only) ------------------------------
+            if (nc == 2) {
+                if (issuer) {
+                    wait_bar(bar_v, par);
+                    constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
+                    const uint32_t ak = desc_lo(t_kb, lay.tile) + row0_64, bv = desc_lo(t_v, 16) + row0_128;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        if (kk < ks) umma_ss(tc + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
+                    umma_commit(bar_mma);
+                }
+                wait_mma();
+                if (warp == 1 || warp == 4) {
+                    // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
+                    // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
+                    const float d = dec[(warp == 1 ? 0 : 32) + lane];
+                    uint8_t* st = bp + (warp == 1 ? lay.s_fwd : lay.s_bwd);
+#pragma unroll
+                    for (int hb = 0; hb < 2; ++hb) {
+                        uint32_t r[32];
+                        tmem_ld32(rc + 64 + hb * 32, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) o[e] = pack_bf16(as_f(r[ch * 8 + 2 * e]) * d, as_f(r[ch * 8 + 2 * e + 1]) * d);
+                            *reinterpret_cast<uint4*>(st + sw_off<128>(lane, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                    fence_async_smem();
+                }
+            }
+        }
+        if (nc == 2) {   // the two chunks exchange their states
+            tc_fence_before();
+            __syncthreads();
+            tc_fence_after();
+        }
+
+        if (chunk_on) {
+            // ---- out = (P v + q~ S_in) / 2 ------------------------------------------------------------------------
+            if (issuer) {
+                wait_bar(bar_v, par);
+                constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
+                uint32_t acc = 0;
+                if (nc == 2) {
+                    // chunk 1 receives the forward state of chunk 0, chunk 0 the backward state of chunk 1
+                    const uint32_t qa = desc_lo(c == 1 ? t_qf : t_qb, 16) + row0_64;
+                    const uint32_t sa = desc_lo(base + (c == 1 ? lay.s_fwd : lay.s_bwd), 16);
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) umma_ss(tc + 64, desc64(qa + kk * 2, kHiK64), desc64(sa + kk * 128, kHiV128), kIdO, kk > 0);
+                    acc = 1;
+                }
+                const uint32_t bv = desc_lo(t_v, 16) + row0_128;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    if (kk < ks) {
+                        umma_ts(tc + 64, tc + kk * 8, desc64(bv + kk * 128, kHiV128), kIdO, kk > 0 ? 1u : acc);
                     }
                 }
                 umma_commit(bar_mma);
             }
-            if (!wait_mma()) timed_out = true;
-        }
-        if (!timed_out) {
+            wait_mma();
             // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
             if (warp_live) {
 #pragma unroll
@@ -513,31 +559,43 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
             }
-            fence_async_smem();
-            tc_fence_before();
-            __syncthreads();
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        // every MMA of this unit has completed and every thread has left its tiles: block-uniform decisions
+        const bool timed_out = *time_flag != 0;
+        const bool slow = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) != 0;
+        if (timed_out) break;
+        if (!slow) {
             if (tid == 0) {
                 tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (has_next) load_gates_qk(unit + (int)gridDim.x);   // these tiles are free already
+                v_load_pending = has_next;   // the v tile only once the store has read it: see above
+            }
+        } else {
+            // A gate left the range the factorised tiles can represent: evaluate this unit by the recurrence
+            // (its scratch overlays the tiles, so the next loads wait until it is done).
+            const size_t ok = (size_t)unit * L * DK, ov = (size_t)unit * L * DV;
+            recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
+                                           args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));
+            fence_async_smem();
+            __syncthreads();
+            if (tid == 0 && has_next) {
+                load_gates_qk(unit + (int)gridDim.x);
+                load_v(unit + (int)gridDim.x);
             }
         }
     }
 
-    // ---- release TMEM (every tcgen05 operation of this block has completed or was never issued) ----
+    if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
+    // ---- release TMEM (every tcgen05 operation of this block has completed) ----
     tc_fence_before();
     __syncthreads();
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols));
-    if (timed_out) {
-        if (tid == 0) atomicOr(args.dev_status, kDevStatusTimeout);
-        return;
-    }
-    if (slow) {
-        // A gate left the range the factorised tiles can represent: evaluate this unit by the recurrence.
-        const size_t ok = (size_t)unit * L * DK, ov = (size_t)unit * L * DV;
-        recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
-                                       args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));
-    }
+    if (tid == 0 && *time_flag != 0) atomicOr(args.dev_status, kDevStatusTimeout);
 }
 
 template <int DK, int DV>
@@ -551,9 +609,12 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
         !make_map(&tv, v, units, L, DV, 64, rows) || !make_map(&to, out, units, L, DV, 64, rows))
         return cudaErrorInvalidValue;
     UArgs a{};
-    a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows;
+    a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows; a.units = units;
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return cudaErrorUnknown;
     // The MMAs of chunk 1 read 128 rows of the operand tiles from row 128 on, i.e. up to (256 - rows) * 64
     // bytes past the last q-type tile: that lands in the v tile, inside the allocation.
     size_t smem = make_layout(rows).total + 1024;   // slack for the manual 1 KB alignment
@@ -561,7 +622,9 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     if (smem < rec) smem = rec;
     cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    bigla_umma_kernel<DK, DV><<<(unsigned)units, kThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
+    // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...
+    const long long grid = units < 2LL * sms ? units : 2LL * sms;
+    bigla_umma_kernel<DK, DV><<<(unsigned)grid, kThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
     count_launch();
     return cudaGetLastError();
 }

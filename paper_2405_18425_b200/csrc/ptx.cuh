@@ -28,13 +28,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after about a quarter of a second and reports it.
+// Bounded wait: polls without backing off for the first few microseconds (the common case: an MMA
+// batch or a TMA load in flight), then sleeps between polls; gives up after about a quarter of a
+// second and reports it.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
     for (uint32_t spin = 0; spin < (1u << 21); ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (spin > 64) __nanosleep(128);
+        if (spin > 4096) __nanosleep(128);
     }
     return false;
+}
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int x, int y, int z) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(y), "r"(z)
+                 : "memory");
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
     asm volatile(
