@@ -106,8 +106,8 @@ struct ULayout {
     uint32_t zf, zb;   // 0/1 tiles of the prefix / suffix sums
     uint32_t s_fwd;    // bf16 state entering chunk 1 from the left  [32][64] (128B swizzle)
     uint32_t s_bwd;    // bf16 state entering chunk 0 from the right
-    uint32_t dec;      // [2][32] fp32 chunk decay factors e^{b_last} (fwd, chunk 0), e^{e_first} (bwd, chunk 1)
-    uint32_t misc;     // five mbarriers, TMEM slot, flags
+    uint32_t dec;      // [2][32] fp32 chunk totals of the log gates: b at the last row of chunk 0, e at the first row of chunk 1
+    uint32_t misc;     // six mbarriers, TMEM slot, flags
     uint32_t total;
 };
 __host__ __device__ inline ULayout make_layout(int rows) {
@@ -191,13 +191,16 @@ constexpr uint32_t kHiV128 = desc_hi(1024, 2);   // MN-major tile with 128-byte 
 constexpr uint32_t kHiZ = desc_hi(256, 0);       // 0/1 tiles, no swizzle
 
 // 1 / x for a normal, positive x without the special-function unit: a bit-level first guess (within 5.1 %)
-// and two Newton steps (relative error below 1e-5).
+// and Newton steps (one: relative error below 0.26 %, two: below 1e-5).  The result only scales bf16
+// operands (rounding unit 0.39 %).
+template <int STEPS>
 __device__ __forceinline__ float fast_rcp(float x) {
     float r = __uint_as_float(0x7EF311C7u - __float_as_uint(x));
-    r = r * fmaf(-x, r, 2.0f);
-    r = r * fmaf(-x, r, 2.0f);
+#pragma unroll
+    for (int i = 0; i < STEPS; ++i) r = r * fmaf(-x, r, 2.0f);
     return r;
 }
+constexpr int kRcpSteps = 2;
 
 template <int DK, int DV>
 __global__ void __launch_bounds__(kThreads, 2)
@@ -218,15 +221,17 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
     const bool row_live = row < L;
     const bool chunk_on = c < nc;
-    const bool issuer = tid == c * kChunk;             // one thread per chunk issues that chunk's MMAs
+    const bool issuer = tid == c * kChunk;             // one thread per chunk issues that chunk's MMAs (thread 0 also the prefix sums)
     const int ks = chunk_on ? (min(L - c * kChunk, kChunk) + 15) >> 4 : 0;   // 16-token K steps of this chunk
     const int nkeys = ks * 16;
-    // mbarriers: log-gate tiles landed, q and k landed, v landed, MMA batches of chunk 0 / chunk 1
+    // mbarriers: log-gate tiles landed, q and k landed, v landed, MMA batches of chunk 0 / chunk 1, prefix sums done
     const uint32_t bar_g = base + lay.misc, bar_qk = bar_g + 8, bar_v = bar_g + 16, bar_mma = bar_g + 24 + 8 * c;
-    const uint32_t slot = bar_g + 40;
-    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 40);
-    volatile int* time_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 44);
-    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 48);   // [4]: (chunk, first / last row) range checks
+    const uint32_t bar_pfx = bar_g + 40, slot = bar_g + 48;
+    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 48);
+    volatile int* time_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 52);
+    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 56);   // [4]: (chunk, first / last row) range checks
+    const int ks_c1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;                          // K steps of chunk 1
+    const int npass_c1 = ks_c1 > 4 ? 2 : 1;
     float* dec = reinterpret_cast<float*>(bp + lay.dec);
     uint32_t mma_phase = 0;
 
@@ -248,7 +253,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
+        for (int i = 0; i < 6; ++i) mbar_init(bar_g + 8 * i, 1);
         *time_flag = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) slow_slot[i] = 0;
@@ -292,6 +297,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t tmem = *slot_p;
     const uint32_t tc = tmem + (uint32_t)c * 128;                   // this chunk's 128 TMEM columns
     const uint32_t rc = tc + ((uint32_t)(wq * 32) << 16);           // ... at this thread's lane
+    const uint32_t rl = tmem + ((uint32_t)(wq * 32) << 16);         // TMEM block 0 at this thread's lane
 
     // A bounded wait that expires raises the flag and lets the block finish the unit on whatever it has:
     // every later wait is bounded too, nothing more is stored, and the host sees the device status word.
@@ -313,7 +319,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
-    bool v_load_pending = false;   // thread 0: the v tile of the current unit has not been requested yet
+    bool v_load_pending = false;      // thread 0: the v tile of the current unit has not been requested yet
+    bool next_loads_issued = false;   // thread 0: the operand tiles of the next unit are already on their way
     for (long long unit_ll = blockIdx.x; unit_ll < args.units; unit_ll += gridDim.x, ++it) {
         const int unit = (int)unit_ll;
         const uint32_t par = it & 1;
@@ -329,47 +336,55 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
 
         if (chunk_on) {
-            // ---- prefix / suffix sums of the log gates -> columns [0,32) / [32,64) of the chunk's TMEM block ----
-            wait_bar(bar_g, par);
-            if (issuer) {
-                constexpr uint32_t kIdS = instr_desc(128, 32, 0, 1);
+            // ---- prefix / suffix sums of the log gates, both chunks at once: B stacks the two chunks' rows along N ----
+            // columns of TMEM block 0:  [0,32) b of chunk 0,  [32,64) b of chunk 1,  [64,96) e of chunk 0,  [96,128) e of chunk 1
+            if (tid == 0) {
+                wait_bar(bar_g, par);
                 const uint32_t zf = desc_lo(base + lay.zf, 128), zb = desc_lo(base + lay.zb, 128);
-                const uint32_t gf = desc_lo(t_qf, 16) + row0_64, gb = desc_lo(t_qb, 16) + row0_64;
+                const uint32_t gf = desc_lo(t_qf, kChunk * 64), gb = desc_lo(t_qb, kChunk * 64);   // second N block = chunk 1's rows
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     if (j < ks) {
                         const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                        umma_ss(tc + 0, desc64(zf + win, kHiZ), desc64(gf + j * 64, kHiK64), kIdS, j > 0);
-                        umma_ss(tc + 32, desc64(zb + win, kHiZ), desc64(gb + j * 64, kHiK64), kIdS, j > 0);
+                        const uint32_t ids = instr_desc(128, j < ks_c1 ? 64 : 32, 0, 1);   // beyond chunk 1's rows: chunk 0 alone
+                        umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(gf + j * 64, kHiK64), ids, j > 0);
+                        umma_ss(tmem + 64, desc64(zb + win, kHiZ), desc64(gb + j * 64, kHiK64), ids, j > 0);
                     }
                 }
-                umma_commit(bar_mma);
+                umma_commit(bar_pfx);
             }
-            wait_mma();
+            wait_bar(bar_pfx, par);
+            tc_fence_after();
             wait_bar(bar_qk, par);
 
             // ---- scaled operands, in place: every thread rewrites its own row ---------------------------------
             if (warp_live) {
                 uint32_t pf[32], pb[32];
-                tmem_ld32(rc, pf);
-                tmem_ld32(rc + 32, pb);
+                tmem_ld32(rl + 32 * c, pf);
+                tmem_ld32(rl + 64 + 32 * c, pb);
                 tc_wait_ld();
+                if (c == 1) {   // chunk 0 may overwrite its TMEM block (where these sums live) from here on
+                    tc_fence_before();
+                    asm volatile("bar.arrive 3, 256;" ::: "memory");
+                }
                 if (row_live) {
                     const int last_row = min(L, (c + 1) * kChunk) - 1;
                     if (row == last_row || row == c * kChunk) {
-                        // b is smallest at the last row of the chunk, e at its first row
-                        float mf = 0.f, mb = 0.f;
+                        // b is smallest at the last row of the chunk, e at its first row (tree minima: these two
+                        // threads hold their whole warps up)
+                        float mf[4] = {0.f, 0.f, 0.f, 0.f}, mb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int d = 0; d < DK; ++d) { mf = fminf(mf, as_f(pf[d])); mb = fminf(mb, as_f(pb[d])); }
-                        if (row == last_row) slow_slot[2 * c + 1] = mf < -kGateRange ? 1 : 0;
-                        if (row == c * kChunk) slow_slot[2 * c] = mb < -kGateRange ? 1 : 0;
-                        if (nc == 2 && row == kChunk - 1) {
+                        for (int d = 0; d < DK; ++d) { mf[d & 3] = fminf(mf[d & 3], as_f(pf[d])); mb[d & 3] = fminf(mb[d & 3], as_f(pb[d])); }
+                        const float mfa = fminf(fminf(mf[0], mf[1]), fminf(mf[2], mf[3])), mba = fminf(fminf(mb[0], mb[1]), fminf(mb[2], mb[3]));
+                        if (row == last_row) slow_slot[2 * c + 1] = mfa < -kGateRange ? 1 : 0;
+                        if (row == c * kChunk) slow_slot[2 * c] = mba < -kGateRange ? 1 : 0;
+                        // chunk totals of the log gates for the state hand-over: b at the last row of chunk 0, e at the first row of chunk 1
+                        if (nc == 2 && (row == kChunk - 1 || row == kChunk)) {
+                            uint4* dst = reinterpret_cast<uint4*>(dec + (row == kChunk ? 32 : 0));
 #pragma unroll
-                            for (int d = 0; d < 32; ++d) dec[d] = ex2(as_f(pf[d]) * kLog2e);
-                        }
-                        if (row == kChunk) {
-#pragma unroll
-                            for (int d = 0; d < 32; ++d) dec[32 + d] = ex2(as_f(pb[d]) * kLog2e);
+                            for (int x = 0; x < 8; ++x)
+                                dst[x] = row == kChunk ? make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3])
+                                                       : make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
                         }
                     }
 #pragma unroll
@@ -385,9 +400,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             const float ex0 = ex2(as_f(pf[8 * ch + 2 * m]) * kLog2e), ex1 = ex2(as_f(pf[8 * ch + 2 * m + 1]) * kLog2e);
                             const float ey0 = ex2(as_f(pb[8 * ch + 2 * m]) * kLog2e), ey1 = ex2(as_f(pb[8 * ch + 2 * m + 1]) * kLog2e);
                             qf[m] = mul_bf16x2(qv[m], pack_bf16(ex0, ex1));                        // q~> = q e^{b}
-                            kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp(ex0), fast_rcp(ex1)));    // k~> = k e^{-b}
+                            kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
                             qb[m] = mul_bf16x2(qv[m], pack_bf16(ey0, ey1));                        // q~< = q e^{e}
-                            kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp(ey0), fast_rcp(ey1)));    // k~< = k e^{-e}
+                            kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
                         }
                         *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
                         *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
@@ -396,8 +411,18 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
             }
+            if (c == 1 && !warp_live) {   // warps of chunk 1 without tokens read no sums but still take part in the hand-over
+                asm volatile("bar.arrive 3, 256;" ::: "memory");
+            }
             fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
-            chunk_handover();
+            if (c == 0 && nc == 2) {
+                // chunk 0's own hand-over, extended by the arrival of chunk 1's warps (they have read their sums)
+                tc_fence_before();
+                named_bar(3, 2 * kChunk);
+                tc_fence_after();
+            } else {
+                chunk_handover();
+            }
             if (tid == 0 && v_load_pending) {
                 // The store of the previous unit was issued a phase ago and has read the v tile by now: this
                 // wait is short, and the tile is only needed again when the chunk summaries are formed.
@@ -478,7 +503,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (warp == 1 || warp == 4) {
                     // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
                     // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
-                    const float d = dec[(warp == 1 ? 0 : 32) + lane];
+                    const float d = ex2(dec[(warp == 1 ? 0 : 32) + lane] * kLog2e);   // decay of the whole chunk for key dim `lane`
                     uint8_t* st = bp + (warp == 1 ? lay.s_fwd : lay.s_bwd);
 #pragma unroll
                     for (int hb = 0; hb < 2; ++hb) {
@@ -527,6 +552,16 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
+            if (tid == 0 && has_next) {
+                // Every MMA that reads the four operand tiles is done once chunk 1's last batch is: the tiles of
+                // the next unit can start to load under the epilogue and the store (unless this unit must be
+                // redone by the recurrence, whose scratch overlays them).
+                if (nc == 2) wait_bar(bar_mma + 8, ((it + 1) * (uint32_t)(npass_c1 + 2) - 1) & 1);
+                if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
+                    load_gates_qk(unit + (int)gridDim.x);
+                    next_loads_issued = true;
+                }
+            }
             // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
             if (warp_live) {
 #pragma unroll
@@ -572,7 +607,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (tid == 0) {
                 tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                if (has_next) load_gates_qk(unit + (int)gridDim.x);   // these tiles are free already
+                if (has_next && !next_loads_issued) load_gates_qk(unit + (int)gridDim.x);
+                next_loads_issued = false;
                 v_load_pending = has_next;   // the v tile only once the store has read it: see above
             }
         } else {
