@@ -221,7 +221,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
     const bool row_live = row < L;
     const bool chunk_on = c < nc;
-    const bool issuer = tid == c * kChunk;             // one thread per chunk issues that chunk's MMAs (thread 0 also the prefix sums)
+    // One thread per chunk issues that chunk's MMAs; the one of chunk 0 also drives the loads and stores.  They sit in
+    // warps 1 and 5, away from the warps whose first / last rows carry the range checks.
+    const bool issuer = tid == c * kChunk + 32;
+    const bool ctl = tid == 32;
     const int ks = chunk_on ? (min(L - c * kChunk, kChunk) + 15) >> 4 : 0;   // 16-token K steps of this chunk
     const int nkeys = ks * 16;
     // mbarriers: log-gate tiles landed, q and k landed, v landed, MMA batches of chunk 0 / chunk 1, prefix sums done
@@ -232,6 +235,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 56);   // [4]: (chunk, first / last row) range checks
     const int ks_c1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;                          // K steps of chunk 1
     const int npass_c1 = ks_c1 > 4 ? 2 : 1;
+    const int ks_c0 = (min(L, kChunk) + 15) >> 4;                                     // K steps of chunk 0
     float* dec = reinterpret_cast<float*>(bp + lay.dec);
     uint32_t mma_phase = 0;
 
@@ -253,7 +257,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     if (tid == 0) {
 #pragma unroll
-        for (int i = 0; i < 6; ++i) mbar_init(bar_g + 8 * i, 1);
+        for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
+        mbar_init(bar_pfx, (uint32_t)nc);   // one commit per chunk issuer
         *time_flag = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) slow_slot[i] = 0;
@@ -319,13 +324,13 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
-    bool v_load_pending = false;      // thread 0: the v tile of the current unit has not been requested yet
-    bool next_loads_issued = false;   // thread 0: the operand tiles of the next unit are already on their way
+    bool v_load_pending = false;      // control thread: the v tile of the current unit has not been requested yet
+    bool next_loads_issued = false;   // control thread: the operand tiles of the next unit are already on their way
     for (long long unit_ll = blockIdx.x; unit_ll < args.units; unit_ll += gridDim.x, ++it) {
         const int unit = (int)unit_ll;
         const uint32_t par = it & 1;
         const bool has_next = unit_ll + gridDim.x < args.units;
-        if (tid == 32 && has_next) {
+        if (tid == 224 && has_next) {
             // pull the tiles of this block's next unit into L2
             const int pu = unit + (int)gridDim.x;
             tma_prefetch_3d(&tm_f, 0, 0, pu);
@@ -338,17 +343,21 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (chunk_on) {
             // ---- prefix / suffix sums of the log gates, both chunks at once: B stacks the two chunks' rows along N ----
             // columns of TMEM block 0:  [0,32) b of chunk 0,  [32,64) b of chunk 1,  [64,96) e of chunk 0,  [96,128) e of chunk 1
-            if (tid == 0) {
+            if (issuer) {
                 wait_bar(bar_g, par);
-                const uint32_t zf = desc_lo(base + lay.zf, 128), zb = desc_lo(base + lay.zb, 128);
-                const uint32_t gf = desc_lo(t_qf, kChunk * 64), gb = desc_lo(t_qb, kChunk * 64);   // second N block = chunk 1's rows
+                // chunk 0's issuer takes the forward sums, chunk 1's the backward sums (a single chunk: both)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (j < ks) {
-                        const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                        const uint32_t ids = instr_desc(128, j < ks_c1 ? 64 : 32, 0, 1);   // beyond chunk 1's rows: chunk 0 alone
-                        umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(gf + j * 64, kHiK64), ids, j > 0);
-                        umma_ss(tmem + 64, desc64(zb + win, kHiZ), desc64(gb + j * 64, kHiK64), ids, j > 0);
+                for (int dir = 0; dir < 2; ++dir) {
+                    if (nc == 2 && dir != c) continue;
+                    const uint32_t z = desc_lo(base + (dir == 0 ? lay.zf : lay.zb), 128);
+                    const uint32_t g = desc_lo(dir == 0 ? t_qf : t_qb, kChunk * 64);   // second N block = chunk 1's rows
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (j < ks_c0) {
+                            const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+                            const uint32_t ids = instr_desc(128, j < ks_c1 ? 64 : 32, 0, 1);   // beyond chunk 1's rows: chunk 0 alone
+                            umma_ss(tmem + 64 * dir, desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
+                        }
                     }
                 }
                 umma_commit(bar_pfx);
@@ -359,56 +368,73 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
             // ---- scaled operands, in place: every thread rewrites its own row ---------------------------------
             if (warp_live) {
-                uint32_t pf[32], pb[32];
-                tmem_ld32(rl + 32 * c, pf);
-                tmem_ld32(rl + 64 + 32 * c, pb);
+                constexpr int kHalves = (DK + 15) / 16;
+                const int last_row = min(L, (c + 1) * kChunk) - 1;
+                const bool check_row = row_live && (row == last_row || row == c * kChunk);
+                float mfa = 0.f, mba = 0.f;
+                uint32_t pf[kHalves][16], pb[kHalves][16];
+                tmem_ld16(rl + 32 * c, pf[0]);
+                tmem_ld16(rl + 64 + 32 * c, pb[0]);
                 tc_wait_ld();
-                if (c == 1) {   // chunk 0 may overwrite its TMEM block (where these sums live) from here on
-                    tc_fence_before();
-                    asm volatile("bar.arrive 3, 256;" ::: "memory");
+                if (kHalves == 2) {   // the second half travels while the first is worked on
+                    tmem_ld16(rl + 32 * c + 16, pf[kHalves - 1]);
+                    tmem_ld16(rl + 64 + 32 * c + 16, pb[kHalves - 1]);
                 }
-                if (row_live) {
-                    const int last_row = min(L, (c + 1) * kChunk) - 1;
-                    if (row == last_row || row == c * kChunk) {
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) {
+                    if (hf == 1) tc_wait_ld();
+                    if (hf == kHalves - 1 && c == 1) {   // chunk 0 may overwrite its TMEM block (where these sums live) from here on
+                        tc_fence_before();
+                        asm volatile("bar.arrive 3, 256;" ::: "memory");
+                    }
+                    if (check_row) {
                         // b is smallest at the last row of the chunk, e at its first row (tree minima: these two
                         // threads hold their whole warps up)
                         float mf[4] = {0.f, 0.f, 0.f, 0.f}, mb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int d = 0; d < DK; ++d) { mf[d & 3] = fminf(mf[d & 3], as_f(pf[d])); mb[d & 3] = fminf(mb[d & 3], as_f(pb[d])); }
-                        const float mfa = fminf(fminf(mf[0], mf[1]), fminf(mf[2], mf[3])), mba = fminf(fminf(mb[0], mb[1]), fminf(mb[2], mb[3]));
-                        if (row == last_row) slow_slot[2 * c + 1] = mfa < -kGateRange ? 1 : 0;
-                        if (row == c * kChunk) slow_slot[2 * c] = mba < -kGateRange ? 1 : 0;
+                        for (int d = 0; d < 16; ++d) { mf[d & 3] = fminf(mf[d & 3], as_f(pf[hf][d])); mb[d & 3] = fminf(mb[d & 3], as_f(pb[hf][d])); }
+                        mfa = fminf(mfa, fminf(fminf(mf[0], mf[1]), fminf(mf[2], mf[3])));
+                        mba = fminf(mba, fminf(fminf(mb[0], mb[1]), fminf(mb[2], mb[3])));
                         // chunk totals of the log gates for the state hand-over: b at the last row of chunk 0, e at the first row of chunk 1
                         if (nc == 2 && (row == kChunk - 1 || row == kChunk)) {
-                            uint4* dst = reinterpret_cast<uint4*>(dec + (row == kChunk ? 32 : 0));
+                            uint4* dst = reinterpret_cast<uint4*>(dec + (row == kChunk ? 32 : 0) + 16 * hf);
 #pragma unroll
-                            for (int x = 0; x < 8; ++x)
-                                dst[x] = row == kChunk ? make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3])
-                                                       : make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
+                            for (int x = 0; x < 4; ++x)
+                                dst[x] = row == kChunk ? make_uint4(pb[hf][4 * x], pb[hf][4 * x + 1], pb[hf][4 * x + 2], pb[hf][4 * x + 3])
+                                                       : make_uint4(pf[hf][4 * x], pf[hf][4 * x + 1], pf[hf][4 * x + 2], pf[hf][4 * x + 3]);
                         }
                     }
+                    if (row_live) {
 #pragma unroll
-                    for (int ch = 0; ch < DK / 8; ++ch) {
-                        const uint32_t off = sw_off<64>(row, ch);
-                        const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
-                        const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + lay.tile + off);
-                        const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w}, kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
-                        uint32_t qf[4], kf[4], qb[4], kb[4];
+                        for (int c8 = 0; c8 < 2; ++c8) {
+                            const int ch = 2 * hf + c8;   // 16-byte chunk of the row: key dims 8 ch .. 8 ch + 7
+                            if (ch >= DK / 8) break;
+                            const uint32_t off = sw_off<64>(row, ch);
+                            const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
+                            const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + lay.tile + off);
+                            const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w}, kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
+                            uint32_t qf[4], kf[4], qb[4], kb[4];
 #pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            // e^{b} on the special-function unit, e^{-b} as its reciprocal on the FMA pipe
-                            const float ex0 = ex2(as_f(pf[8 * ch + 2 * m]) * kLog2e), ex1 = ex2(as_f(pf[8 * ch + 2 * m + 1]) * kLog2e);
-                            const float ey0 = ex2(as_f(pb[8 * ch + 2 * m]) * kLog2e), ey1 = ex2(as_f(pb[8 * ch + 2 * m + 1]) * kLog2e);
-                            qf[m] = mul_bf16x2(qv[m], pack_bf16(ex0, ex1));                        // q~> = q e^{b}
-                            kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
-                            qb[m] = mul_bf16x2(qv[m], pack_bf16(ey0, ey1));                        // q~< = q e^{e}
-                            kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
+                            for (int m = 0; m < 4; ++m) {
+                                // e^{b} on the special-function unit, e^{-b} as its reciprocal on the FMA pipe
+                                const int d0 = 8 * c8 + 2 * m;
+                                const float ex0 = ex2(as_f(pf[hf][d0]) * kLog2e), ex1 = ex2(as_f(pf[hf][d0 + 1]) * kLog2e);
+                                const float ey0 = ex2(as_f(pb[hf][d0]) * kLog2e), ey1 = ex2(as_f(pb[hf][d0 + 1]) * kLog2e);
+                                qf[m] = mul_bf16x2(qv[m], pack_bf16(ex0, ex1));                                              // q~> = q e^{b}
+                                kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
+                                qb[m] = mul_bf16x2(qv[m], pack_bf16(ey0, ey1));                                              // q~< = q e^{e}
+                                kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
+                            }
+                            *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+                            *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
+                            *reinterpret_cast<uint4*>(bp + 3 * lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
+                            *reinterpret_cast<uint4*>(bp + 0 * lay.tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
                         }
-                        *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
-                        *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
-                        *reinterpret_cast<uint4*>(bp + 3 * lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
-                        *reinterpret_cast<uint4*>(bp + 0 * lay.tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
                     }
+                }
+                if (check_row) {
+                    if (row == last_row) slow_slot[2 * c + 1] = mfa < -kGateRange ? 1 : 0;
+                    if (row == c * kChunk) slow_slot[2 * c] = mba < -kGateRange ? 1 : 0;
                 }
             }
             if (c == 1 && !warp_live) {   // warps of chunk 1 without tokens read no sums but still take part in the hand-over
@@ -423,7 +449,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             } else {
                 chunk_handover();
             }
-            if (tid == 0 && v_load_pending) {
+            if (ctl && v_load_pending) {
                 // The store of the previous unit was issued a phase ago and has read the v tile by now: this
                 // wait is short, and the tile is only needed again when the chunk summaries are formed.
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -552,7 +578,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
-            if (tid == 0 && has_next) {
+            if (ctl && has_next) {
                 // Every MMA that reads the four operand tiles is done once chunk 1's last batch is: the tiles of
                 // the next unit can start to load under the epilogue and the store (unless this unit must be
                 // redone by the recurrence, whose scratch overlays them).
@@ -604,7 +630,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const bool slow = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) != 0;
         if (timed_out) break;
         if (!slow) {
-            if (tid == 0) {
+            if (ctl) {
                 tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 if (has_next && !next_loads_issued) load_gates_qk(unit + (int)gridDim.x);
@@ -619,14 +645,14 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                            args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));
             fence_async_smem();
             __syncthreads();
-            if (tid == 0 && has_next) {
+            if (ctl && has_next) {
                 load_gates_qk(unit + (int)gridDim.x);
                 load_v(unit + (int)gridDim.x);
             }
         }
     }
 
-    if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
+    if (ctl) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
     // ---- release TMEM (every tcgen05 operation of this block has completed) ----
     tc_fence_before();
     __syncthreads();
