@@ -492,14 +492,17 @@ bool mma_supported(int dk, int dv) {
 size_t mma_workspace_bytes(long long units, int L, int dk, int dv) {
     const Plan pl = make_plan(L);
     if (pl.nseg == 1) return 0;
+    if (kernel_preference() != VIG_KERNEL_MMA_SYNC) return umma_long_workspace_bytes(units, L, dk, dv);
     return ws_layout(units, pl.nseg, dv, (dk + 15) / 16 * 16).total;
 }
 
 cudaError_t launch_bigla_mma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                              const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
                              int L, int dk, int dv, void* ws, cudaStream_t stream) {
-    if (kernel_preference() != VIG_KERNEL_MMA_SYNC && umma_supported(dk, dv, L))
-        return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, stream);
+    if (kernel_preference() != VIG_KERNEL_MMA_SYNC) {
+        if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, stream);
+        return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
+    }
 #define VIG_CASE(DK_, DV_) \
     if (dk == DK_ && dv == DV_) return launch_t<DK_, DV_>(q, k, v, la_f, la_b, out, units, L, ws, stream);
     VIG_CASE(16, 32) VIG_CASE(16, 48) VIG_CASE(16, 64)

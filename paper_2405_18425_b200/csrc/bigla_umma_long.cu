@@ -1,0 +1,598 @@
+// bf16 BiGLA forward for sequences longer than one thread block holds, on tcgen05 / TMEM.
+//
+// The sequence of every (batch, head) unit is cut into chunks of 128 tokens; a task is one chunk, and the
+// running states of Eq. 6 that cross chunk boundaries travel through scratch memory in three launches:
+//   1. summary: per chunk, the state a zero input would leave behind, U> = diag(e^{b_last}) (k~>)^T v and
+//      U< = diag(e^{e_first}) (k~<)^T v, and the chunk's decay d> = e^{b_last}, d< = e^{e_first}
+//      (b, e: prefix / suffix sums of the log gates inside the chunk, as in the single-block kernel);
+//   2. fold: S>_in(m + 1) = d>(m) S>_in(m) + U>(m) from the left, S<_in(m - 1) = d<(m) S<_in(m) + U<(m) from the
+//      right, in fp32; every incoming state is written back over its summary as the bf16 shared-memory image
+//      the next launch copies in with one bulk copy;
+//   3. main: per chunk, out = ( P v + q~> S>_in + q~< S<_in ) / 2 with P = tril(q~> k~>^T) + triu(q~< k~<^T).
+// Blocks are persistent (three per SM, 128 threads, 128 TMEM columns each) and walk over the tasks; thread r
+// owns token r of the chunk in every element-wise phase.  All products are tcgen05.mma with M = 128.
+#include <cuda.h>
+
+#include "recurrence.cuh"
+#include "tma_host.h"
+#include "umma.cuh"
+#include "vig_internal.h"
+
+namespace vig {
+namespace {
+
+using namespace umma;
+
+constexpr int kLThreads = 128;
+constexpr uint32_t kLTmemCols = 128;
+constexpr int kLBlocksPerSm = 3;
+enum LongMode { kLMain = 0, kLSummary = 1 };
+
+// ---- scratch ---------------------------------------------------------------------------------------------
+// slot(unit, chunk, dir): 32 x DV fp32 (summary, key dim major), overwritten by the fold with a 4 KB bf16 tile
+// image [32][64] (128-byte rows, 128B swizzle);  decay(unit, chunk, dir): 32 fp32;  flags(unit): int.
+struct LongWs {
+    size_t slot_bytes, decay_off, flags_off, total;
+};
+LongWs long_ws_layout(long long units, int nch, int dv) {
+    LongWs w;
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    w.slot_bytes = (size_t)32 * dv * 4 < 4096 ? 4096 : (size_t)32 * dv * 4;
+    w.decay_off = up((size_t)units * nch * 2 * w.slot_bytes);
+    w.flags_off = w.decay_off + up((size_t)units * nch * 2 * 32 * 4);
+    w.total = w.flags_off + up((size_t)units * 4);
+    return w;
+}
+
+// ---- shared memory -------------------------------------------------------------------------------------------
+struct LLayout {
+    static constexpr uint32_t tile = 128 * 64;         // q-type tile [128][32] bf16, 64B swizzle; four from offset 0:
+                                                       //   loaded: q, k, log alpha>, log alpha<; scaled: k~<, k~>, q~>, q~<
+    static constexpr uint32_t v = 4 * tile;            // v tile [128][64] bf16 (128B swizzle), later the output tile
+    static constexpr uint32_t zf = v + 128 * 128;
+    static constexpr uint32_t zb = zf + kZBytes;
+    static constexpr uint32_t s_fwd = (zb + kZBytes + 1023u) & ~1023u;   // incoming states, bf16 [32][64], 128B swizzle
+    static constexpr uint32_t s_bwd = s_fwd + 4096;
+    static constexpr uint32_t misc = s_bwd + 4096;     // mbarriers, TMEM slot, flags
+    static constexpr uint32_t total = misc + 128;
+};
+
+struct LArgs {
+    const __nv_bfloat16 *q, *k, *v, *la_f, *la_b;
+    __nv_bfloat16* out;
+    int L, nch;
+    long long tasks;
+    uint8_t* ws_slots;    // [units][nch][2][slot_bytes]
+    float* ws_decay;      // [units][nch][2][32]
+    int* ws_flags;        // [units]
+    uint32_t slot_bytes;
+    int* dev_status;
+};
+
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+template <int DK, int DV, int MODE>
+__global__ void __launch_bounds__(kLThreads, kLBlocksPerSm)
+bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_b,
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const LArgs args) {
+    static_assert((DK == 16 || DK == 24 || DK == 32) && (DV == 32 || DV == 48 || DV == 64), "unsupported head size");
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* bp = smem_raw + (base - smem_u32(smem_raw));
+    using Y = LLayout;
+
+    const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
+    const int L = args.L, nch = args.nch;
+    const bool ctl = tid == 32;   // issues loads, MMAs and stores (warp 1: not a range-check warp)
+    // mbarriers: log gates landed, q / k landed, v landed, incoming states landed, MMA batch done
+    const uint32_t bar_g = base + Y::misc, bar_qk = bar_g + 8, bar_v = bar_g + 16, bar_s = bar_g + 24, bar_mma = bar_g + 32;
+    const uint32_t slot = bar_g + 40;
+    volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + Y::misc + 40);
+    volatile int* time_flag = reinterpret_cast<volatile int*>(bp + Y::misc + 44);
+    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + Y::misc + 48);   // [2]: first-row / last-row range checks
+    float* totals = reinterpret_cast<float*>(bp + Y::s_fwd);   // summary mode: [2][32] chunk totals of the log gates (state tiles unused there)
+    uint32_t mma_phase = 0;
+
+    const uint32_t t_kb = base, t_kf = base + Y::tile, t_qf = base + 2 * Y::tile, t_qb = base + 3 * Y::tile;
+    const uint32_t t_v = base + Y::v;
+
+    auto task_unit = [&](long long t) { return (int)(t / nch); };
+    auto task_chunk = [&](long long t) { return (int)(t % nch); };
+    auto load_operands = [&](long long t) {   // everything but v
+        const int u = task_unit(t), r0 = task_chunk(t) * kChunk;
+        mbar_expect_tx(bar_g, 2 * Y::tile);
+        tma_load_3d(t_qf, &tm_f, 0, r0, u, bar_g);
+        tma_load_3d(t_qb, &tm_b, 0, r0, u, bar_g);
+        if (MODE == kLMain) {
+            mbar_expect_tx(bar_qk, 2 * Y::tile);
+            tma_load_3d(t_kb, &tm_q, 0, r0, u, bar_qk);
+            tma_load_3d(t_kf, &tm_k, 0, r0, u, bar_qk);
+            const uint8_t* sl = args.ws_slots + (size_t)t * 2 * args.slot_bytes;
+            mbar_expect_tx(bar_s, 2 * 4096);
+            bulk_load_1d(base + Y::s_fwd, sl, 4096, bar_s);
+            bulk_load_1d(base + Y::s_bwd, sl + args.slot_bytes, 4096, bar_s);
+        } else {
+            mbar_expect_tx(bar_qk, Y::tile);
+            tma_load_3d(t_kf, &tm_k, 0, r0, u, bar_qk);
+        }
+    };
+    auto load_v = [&](long long t) {
+        mbar_expect_tx(bar_v, 128 * 128);
+        tma_load_3d(t_v, &tm_v, 0, task_chunk(t) * kChunk, task_unit(t), bar_v);
+    };
+
+    if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
+        *time_flag = 0;
+        slow_slot[0] = slow_slot[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (wq == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(kLTmemCols));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
+    }
+    // the 240 rows of the 0/1 tiles, two passes of 128 threads
+    build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid);
+    build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid + kLThreads);
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot_p;
+    const uint32_t rc = tmem + ((uint32_t)(wq * 32) << 16);   // this thread's TMEM lane
+
+    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
+        if (!mbar_wait_bounded(bar, parity)) *time_flag = 1;
+    };
+    auto wait_mma = [&]() {
+        wait_bar(bar_mma, mma_phase & 1);
+        ++mma_phase;
+        tc_fence_after();
+    };
+    auto handover = [&]() {
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    };
+
+    if (ctl && blockIdx.x < args.tasks) {
+        load_operands(blockIdx.x);
+        load_v(blockIdx.x);
+    }
+
+    uint32_t it = 0;
+    bool v_load_pending = false;   // control thread: the v tile of the current task has not been requested yet
+    for (long long task = blockIdx.x; task < args.tasks; task += gridDim.x, ++it) {
+        const uint32_t par = it & 1;
+        const int unit = task_unit(task), m = task_chunk(task);
+        const long long next = task + gridDim.x;
+        const bool has_next = next < args.tasks;
+        const int rows_here = min(kChunk, L - m * kChunk);
+        const int ks = (rows_here + 15) >> 4, nkeys = ks * 16;
+        const int row = wq * 32 + lane;
+        const bool warp_live = wq * 32 < rows_here, row_live = row < rows_here;
+        // a unit whose gates left the factorised range (found by the summary launch) is redone by the recurrence
+        const bool unit_slow = MODE == kLMain && args.ws_flags[unit] != 0;
+
+        if (tid == 96 && has_next) {   // pull the next task's tiles into L2
+            const int pu = task_unit(next), pr = task_chunk(next) * kChunk;
+            tma_prefetch_3d(&tm_f, 0, pr, pu);
+            tma_prefetch_3d(&tm_b, 0, pr, pu);
+            tma_prefetch_3d(&tm_k, 0, pr, pu);
+            tma_prefetch_3d(&tm_v, 0, pr, pu);
+            if (MODE == kLMain) tma_prefetch_3d(&tm_q, 0, pr, pu);
+        }
+
+        // ---- prefix / suffix sums of the log gates -> TMEM columns [0,32) / [32,64) -----------------------------
+        if (ctl) {
+            wait_bar(bar_g, par);
+            constexpr uint32_t kIdS = instr_desc(128, 32, 0, 1);
+            const uint32_t zf = desc_lo(base + Y::zf, 128), zb = desc_lo(base + Y::zb, 128);
+            const uint32_t gf = desc_lo(t_qf, 16), gb = desc_lo(t_qb, 16);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < ks) {
+                    const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+                    umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(gf + j * 64, kHiK64), kIdS, j > 0);
+                    umma_ss(tmem + 32, desc64(zb + win, kHiZ), desc64(gb + j * 64, kHiK64), kIdS, j > 0);
+                }
+            }
+            umma_commit(bar_mma);
+        }
+        wait_mma();
+        wait_bar(bar_qk, par);
+
+        // ---- scaled operands, in place: every thread rewrites its own row -----------------------------------------
+        if (warp_live) {
+            constexpr int kHalves = (DK + 15) / 16;
+            const bool check_row = row_live && (row == rows_here - 1 || row == 0);
+            float mfa = 0.f, mba = 0.f;
+#pragma unroll
+            for (int hf = 0; hf < kHalves; ++hf) {
+                uint32_t pf[16], pb[16];
+                tmem_ld16(rc + 16 * hf, pf);
+                tmem_ld16(rc + 32 + 16 * hf, pb);
+                tc_wait_ld();
+                if (check_row) {
+                    // b is smallest at the last row of the chunk, e at its first row
+                    float mf[4] = {0.f, 0.f, 0.f, 0.f}, mb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int d = 0; d < 16; ++d) { mf[d & 3] = fminf(mf[d & 3], as_f(pf[d])); mb[d & 3] = fminf(mb[d & 3], as_f(pb[d])); }
+                    mfa = fminf(mfa, fminf(fminf(mf[0], mf[1]), fminf(mf[2], mf[3])));
+                    mba = fminf(mba, fminf(fminf(mb[0], mb[1]), fminf(mb[2], mb[3])));
+                    if (MODE == kLSummary) {
+                        // chunk totals of the log gates: b at the last row, e at the first row
+                        if (row == rows_here - 1) {
+#pragma unroll
+                            for (int x = 0; x < 4; ++x)
+                                reinterpret_cast<uint4*>(totals + 16 * hf)[x] = make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
+                        }
+                        if (row == 0) {
+#pragma unroll
+                            for (int x = 0; x < 4; ++x)
+                                reinterpret_cast<uint4*>(totals + 32 + 16 * hf)[x] = make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3]);
+                        }
+                    }
+                }
+                if (row_live) {
+#pragma unroll
+                    for (int c8 = 0; c8 < 2; ++c8) {
+                        const int ch = 2 * hf + c8;   // 16-byte chunk of the row: key dims 8 ch .. 8 ch + 7
+                        if (ch >= DK / 8) break;
+                        const uint32_t off = sw_off<64>(row, ch);
+                        const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + Y::tile + off);
+                        const uint32_t kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
+                        uint32_t kf[4], kb[4];
+                        if (MODE == kLMain) {
+                            const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
+                            const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w};
+                            uint32_t qf[4], qb[4];
+#pragma unroll
+                            for (int mm = 0; mm < 4; ++mm) {
+                                // e^{b} on the special-function unit, e^{-b} as its reciprocal on the FMA pipe
+                                const int d0 = 8 * c8 + 2 * mm;
+                                const float ex0 = ex2(as_f(pf[d0]) * kLog2e), ex1 = ex2(as_f(pf[d0 + 1]) * kLog2e);
+                                const float ey0 = ex2(as_f(pb[d0]) * kLog2e), ey1 = ex2(as_f(pb[d0 + 1]) * kLog2e);
+                                qf[mm] = mul_bf16x2(qv[mm], pack_bf16(ex0, ex1));                                              // q~> = q e^{b}
+                                kf[mm] = mul_bf16x2(kv[mm], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
+                                qb[mm] = mul_bf16x2(qv[mm], pack_bf16(ey0, ey1));                                              // q~< = q e^{e}
+                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
+                            }
+                            *reinterpret_cast<uint4*>(bp + 2 * Y::tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+                            *reinterpret_cast<uint4*>(bp + 3 * Y::tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
+                        } else {
+#pragma unroll
+                            for (int mm = 0; mm < 4; ++mm) {
+                                const int d0 = 8 * c8 + 2 * mm;
+                                kf[mm] = mul_bf16x2(kv[mm], pack_bf16(ex2(-as_f(pf[d0]) * kLog2e), ex2(-as_f(pf[d0 + 1]) * kLog2e)));
+                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(ex2(-as_f(pb[d0]) * kLog2e), ex2(-as_f(pb[d0 + 1]) * kLog2e)));
+                            }
+                        }
+                        *reinterpret_cast<uint4*>(bp + 1 * Y::tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
+                        *reinterpret_cast<uint4*>(bp + 0 * Y::tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
+                    }
+                }
+            }
+            if (MODE == kLSummary) {
+                // the q tile is not loaded in this mode: rows without tokens and padding key dims of k~< must read as zero
+                if (!row_live || DK < 32) {
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch)
+                        if (!row_live || ch >= DK / 8) *reinterpret_cast<uint4*>(bp + sw_off<64>(row, ch)) = make_uint4(0, 0, 0, 0);
+                }
+            }
+            if (check_row) {
+                if (row == rows_here - 1) slow_slot[1] = mfa < -kGateRange ? 1 : 0;
+                if (row == 0) slow_slot[0] = mba < -kGateRange ? 1 : 0;
+            }
+        } else if (MODE == kLSummary) {
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) *reinterpret_cast<uint4*>(bp + sw_off<64>(row, ch)) = make_uint4(0, 0, 0, 0);
+        }
+        fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
+        handover();
+        if (ctl && v_load_pending) {
+            // the store of the previous task has read the v tile by now; the tile is needed again only further down
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            load_v(task);
+            v_load_pending = false;
+        }
+
+        if constexpr (MODE == kLSummary) {
+            // ---- U = [k~< | k~>]^T v -> TMEM columns [64,128); rows 0..31: backward, rows 32..63: forward ----------
+            if (ctl) {
+                wait_bar(bar_v, par);
+                constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
+                const uint32_t ak = desc_lo(t_kb, Y::tile), bv = desc_lo(t_v, 16);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    if (kk < ks) umma_ss(tmem + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
+                umma_commit(bar_mma);
+            }
+            wait_mma();
+            if (wq < 2) {
+                // lane = key dim; warp 0: backward summary, warp 1: forward summary
+                const int dir = wq == 1 ? 0 : 1;
+                const float d = lane < DK ? ex2(totals[(dir == 0 ? 0 : 32) + lane] * kLog2e) : 1.f;   // decay of the whole chunk for this key dim
+                float* dst = reinterpret_cast<float*>(args.ws_slots + ((size_t)task * 2 + dir) * args.slot_bytes) + (size_t)lane * DV;
+#pragma unroll
+                for (int hb = 0; hb < 2; ++hb) {
+                    if (hb * 32 >= DV) break;
+                    uint32_t r[32];
+                    tmem_ld32(rc + 64 + hb * 32, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        if (hb * 32 + 4 * x < DV)
+                            reinterpret_cast<float4*>(dst + hb * 32)[x] =
+                                make_float4(as_f(r[4 * x]) * d, as_f(r[4 * x + 1]) * d, as_f(r[4 * x + 2]) * d, as_f(r[4 * x + 3]) * d);
+                    }
+                }
+                args.ws_decay[((size_t)task * 2 + dir) * 32 + lane] = d;
+            }
+            handover();
+            if (tid == 0 && (slow_slot[0] | slow_slot[1]) != 0) args.ws_flags[unit] = 1;
+            if (*time_flag != 0) break;
+            if (ctl && has_next) {
+                load_operands(next);
+                load_v(next);
+            }
+        } else {
+        // ---- main mode ---------------------------------------------------------------------------------------------
+        // P, key columns [64 p, 64 p + 64): forward scores -> columns [0,64), backward -> [64,128)
+        uint32_t hold[32];   // packed bf16 P of this row, key columns 0..63
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+            const int n = min(nkeys - 64 * p, 64);
+            if (n <= 0) break;
+            if (ctl) {
+                const uint32_t idp = instr_desc(128, n, 0, 0);
+                const uint32_t aqf = desc_lo(t_qf, 16), aqb = desc_lo(t_qb, 16), bkf = desc_lo(t_kf, 16), bkb = desc_lo(t_kb, 16);
+#pragma unroll
+                for (int kk = 0; kk < 2; ++kk) {
+                    umma_ss(tmem + 0, desc64(aqf + kk * 2, kHiK64), desc64(bkf + p * 256 + kk * 2, kHiK64), idp, kk > 0);
+                    umma_ss(tmem + 64, desc64(aqb + kk * 2, kHiK64), desc64(bkb + p * 256 + kk * 2, kHiK64), idp, kk > 0);
+                }
+                umma_commit(bar_mma);
+            }
+            wait_mma();
+            if (warp_live) {
+                uint32_t pk[16];
+                combine_any(2 * p, wq, true, rc, rc + 64, lane, pk);
+                if (p == 0) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) hold[e] = pk[e];
+                } else {
+                    // key block 2 has been read: columns [0,32) are dead and take the packed first half
+                    uint32_t h0[16], h1[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) { h0[e] = hold[e]; h1[e] = hold[16 + e]; }
+                    tmem_st16(rc, h0);
+                    tmem_st16(rc + 16, h1);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) hold[e] = pk[e];
+                }
+                combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, pk);
+                if (p == 0) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) hold[16 + e] = pk[e];
+                    if (nkeys <= 64) {   // no second half
+                        uint32_t h0[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) h0[e] = hold[e];
+                        tmem_st16(rc, h0);
+                        tmem_st16(rc + 16, pk);
+                    }
+                } else {
+                    uint32_t h0[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) h0[e] = hold[e];
+                    tmem_st16(rc + 32, h0);
+                    tmem_st16(rc + 48, pk);
+                }
+            }
+            tc_wait_st();
+            handover();
+        }
+
+        // out = (q~> S>_in + q~< S<_in + P v) / 2
+        if (ctl) {
+            wait_bar(bar_v, par);
+            wait_bar(bar_s, par);
+            constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
+            const uint32_t qf = desc_lo(t_qf, 16), qb = desc_lo(t_qb, 16);
+            const uint32_t sf = desc_lo(base + Y::s_fwd, 16), sb = desc_lo(base + Y::s_bwd, 16), bv = desc_lo(t_v, 16);
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) umma_ss(tmem + 64, desc64(qf + kk * 2, kHiK64), desc64(sf + kk * 128, kHiV128), kIdO, kk > 0);
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) umma_ss(tmem + 64, desc64(qb + kk * 2, kHiK64), desc64(sb + kk * 128, kHiV128), kIdO, 1);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)
+                if (kk < ks) umma_ts(tmem + 64, tmem + kk * 8, desc64(bv + kk * 128, kHiV128), kIdO, 1);
+            umma_commit(bar_mma);
+        }
+        wait_mma();
+        const bool next_early = has_next && !unit_slow;
+        if (ctl && next_early && *time_flag == 0) load_operands(next);   // every MMA that reads the operand tiles is done
+        if (warp_live) {
+            // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
+#pragma unroll
+            for (int hb = 0; hb < DV / 32; ++hb) {
+                uint32_t r[32];
+                tmem_ld32(rc + 64 + hb * 32, r);
+                tc_wait_ld();
+                if (row_live) {
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(bp + Y::v + sw_off<128>(row, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+            }
+            if (DV == 48) {
+                uint32_t r[16];
+                tmem_ld16(rc + 64 + 32, r);
+                tc_wait_ld();
+                if (row_live) {
+#pragma unroll
+                    for (int ch = 0; ch < 2; ++ch) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(bp + Y::v + sw_off<128>(row, 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+            }
+        }
+        fence_async_smem();
+        handover();
+        if (*time_flag != 0) break;
+        if (!unit_slow) {
+            if (ctl) {
+                tma_store_3d(&tm_o, 0, m * kChunk, unit, t_v);   // rows >= L and columns >= dv are clipped
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                if (has_next && !next_early) load_operands(next);
+                v_load_pending = has_next;   // the v tile only once the store has read it
+            }
+        } else {
+            // the first chunk's task redoes the whole unit by the recurrence (its scratch overlays the tiles, so the
+            // next loads wait until it is done); the other chunks of the unit store nothing
+            if (m == 0) {
+                const size_t ok = (size_t)unit * L * DK, ov = (size_t)unit * L * DV;
+                recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
+                                               args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));
+                fence_async_smem();
+                __syncthreads();
+            }
+            if (ctl && has_next) {
+                load_operands(next);
+                load_v(next);
+            }
+        }
+        }   // main mode
+    }
+
+    if (ctl) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
+    tc_fence_before();
+    __syncthreads();
+    if (wq == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kLTmemCols));
+    if (tid == 0 && *time_flag != 0) atomicOr(args.dev_status, kDevStatusTimeout);
+}
+
+// Sequential fold of the chunk summaries of one unit and direction.  Thread (i, c) owns the eight value dims
+// 8 c .. 8 c + 7 of key dim i.  Chunks are taken in batches of eight so that their loads are all in flight
+// together; after a batch is in registers the incoming states are written, as bf16 tile images, over the
+// first 4 KB of the same slots.
+template <int DV>
+__global__ void __launch_bounds__(32 * (DV / 8))
+bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, const int* ws_flags, int nch, uint32_t slot_bytes) {
+    constexpr int CPR = DV / 8;   // 16-byte chunks of live value dims per row of the image
+    const int unit = blockIdx.x, dir = blockIdx.y;
+    if (ws_flags[unit] != 0) return;
+    const int i = threadIdx.x / CPR, c = threadIdx.x % CPR;
+    float carry[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) carry[e] = 0.f;
+    for (int mb = 0; mb < nch; mb += 8) {
+        float4 u[8][2];
+        float d[8];
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            if (mb + b < nch) {
+                const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
+                const size_t s = ((size_t)unit * nch + m) * 2 + dir;
+                const float4* src = reinterpret_cast<const float4*>(ws_slots + s * slot_bytes) + ((size_t)i * DV + 8 * c) / 4;
+                u[b][0] = src[0];
+                u[b][1] = src[1];
+                d[b] = ws_decay[s * 32 + i];
+            }
+        }
+        __syncthreads();   // every summary of the batch is in registers before any of its slots is overwritten
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            if (mb + b < nch) {
+                const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
+                uint8_t* img = ws_slots + (((size_t)unit * nch + m) * 2 + dir) * slot_bytes;
+                uint4 o;
+                o.x = pack_bf16(carry[0], carry[1]); o.y = pack_bf16(carry[2], carry[3]);
+                o.z = pack_bf16(carry[4], carry[5]); o.w = pack_bf16(carry[6], carry[7]);
+                *reinterpret_cast<uint4*>(img + i * 128 + ((c ^ (i & 7)) << 4)) = o;
+                if (c < 8 - CPR)   // value dims beyond dv read as zero
+                    *reinterpret_cast<uint4*>(img + i * 128 + (((CPR + c) ^ (i & 7)) << 4)) = make_uint4(0, 0, 0, 0);
+                const float uu[8] = {u[b][0].x, u[b][0].y, u[b][0].z, u[b][0].w, u[b][1].x, u[b][1].y, u[b][1].z, u[b][1].w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) carry[e] = fmaf(carry[e], d[b], uu[e]);
+            }
+        }
+        __syncthreads();   // images written before the next batch's loads (they touch other slots, but keep the order plain)
+    }
+}
+
+template <int DK, int DV>
+cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* la_f,
+                          const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units, int L, void* ws,
+                          cudaStream_t stream) {
+    const int nch = (L + kChunk - 1) / kChunk;
+    CUtensorMap tq, tk, tf, tb, tv, to;
+    if (!make_map(&tq, q, units, L, DK, 32, kChunk) || !make_map(&tk, k, units, L, DK, 32, kChunk) ||
+        !make_map(&tf, la_f, units, L, DK, 32, kChunk) || !make_map(&tb, la_b, units, L, DK, 32, kChunk) ||
+        !make_map(&tv, v, units, L, DV, 64, kChunk) || !make_map(&to, out, units, L, DV, 64, kChunk))
+        return cudaErrorInvalidValue;
+    const LongWs wl = long_ws_layout(units, nch, DV);
+    LArgs a{};
+    a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out;
+    a.L = L; a.nch = nch; a.tasks = units * nch;
+    a.ws_slots = static_cast<uint8_t*>(ws);
+    a.ws_decay = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + wl.decay_off);
+    a.ws_flags = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + wl.flags_off);
+    a.slot_bytes = (uint32_t)wl.slot_bytes;
+    a.dev_status = device_status_ptr();
+    if (!a.dev_status) return cudaErrorUnknown;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return cudaErrorUnknown;
+    size_t smem = LLayout::total + 1024;   // slack for the manual 1 KB alignment
+    const size_t rec = (size_t)rec_plan(kLThreads, DK, DV).smem_floats * 4 + 1024;
+    if (smem < rec) smem = rec;
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLSummary>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLMain>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(a.ws_flags, 0, (size_t)units * 4, stream)) != cudaSuccess) return e;
+    const long long cap = (long long)kLBlocksPerSm * sms;
+    const unsigned grid = (unsigned)(a.tasks < cap ? a.tasks : cap);   // persistent blocks: block b takes tasks b, b + grid, ...
+    bigla_long_kernel<DK, DV, kLSummary><<<grid, kLThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
+    bigla_long_fold_kernel<DV><<<dim3((unsigned)units, 2), 32 * (DV / 8), 0, stream>>>(a.ws_slots, a.ws_decay, a.ws_flags, nch, a.slot_bytes);
+    bigla_long_kernel<DK, DV, kLMain><<<grid, kLThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
+    count_launch(3);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t umma_long_workspace_bytes(long long units, int L, int dk, int dv) {
+    (void)dk;
+    return long_ws_layout(units, (L + kChunk - 1) / kChunk, dv).total;
+}
+
+cudaError_t launch_bigla_umma_long(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                   const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
+                                   int L, int dk, int dv, void* ws, cudaStream_t stream) {
+#define VIG_CASE(DK_, DV_) \
+    if (dk == DK_ && dv == DV_) return launch_long_t<DK_, DV_>(q, k, v, la_f, la_b, out, units, L, ws, stream);
+    VIG_CASE(16, 32) VIG_CASE(16, 48) VIG_CASE(16, 64)
+    VIG_CASE(24, 32) VIG_CASE(24, 48) VIG_CASE(24, 64)
+    VIG_CASE(32, 32) VIG_CASE(32, 48) VIG_CASE(32, 64)
+#undef VIG_CASE
+    return cudaErrorNotSupported;
+}
+
+}  // namespace vig

@@ -1,0 +1,176 @@
+// Pieces shared by the tcgen05 BiGLA kernels: tcgen05 / TMEM wrappers, shared-memory and instruction
+// descriptors, the 0/1 tiles of the prefix-sum products, masking and packing of the score tile.
+#pragma once
+#include <cuda.h>
+
+#include "ptx.cuh"
+
+namespace vig {
+namespace umma {
+
+constexpr int kChunk = 128;     // rows per MMA chunk
+constexpr float kGateRange = 60.f;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kZRows = 240;                 // 112 constant rows, 16 triangle rows, 112 constant rows
+constexpr uint32_t kZBytes = kZRows * 32;        // 16 bf16 per row
+
+// ---- tcgen05 wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Instruction descriptor of kind::f16: fp32 accumulate, bf16 A and B, majors, N >> 3, M >> 4.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+}
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t addr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(addr));
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,"
+        "%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(addr));
+}
+__device__ __forceinline__ void tmem_st16(uint32_t addr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(addr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
+
+// Packed bf16 values of one 32-column block of P for this thread's row.  REL < 0: the block lies left
+// of the diagonal block (forward scores only), REL > 0: right of it (backward only), REL == 0: the
+// diagonal block, forward part masked to s <= t, backward part to s >= t, summed in fp32.
+template <int REL>
+__device__ __forceinline__ void combine_block(uint32_t fwd_addr, uint32_t bwd_addr, int lane, uint32_t (&pk)[16]) {
+    if (REL != 0) {
+        uint32_t r[32];
+        tmem_ld32(REL < 0 ? fwd_addr : bwd_addr, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(as_f(r[2 * e]), as_f(r[2 * e + 1]));
+    } else {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t f[16], b[16];
+            tmem_ld16(fwd_addr + 16 * h, f);
+            tmem_ld16(bwd_addr + 16 * h, b);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int s0 = 16 * h + 2 * e, s1 = s0 + 1;
+                const float lo = (s0 <= lane ? as_f(f[2 * e]) : 0.f) + (s0 >= lane ? as_f(b[2 * e]) : 0.f);
+                const float hi = (s1 <= lane ? as_f(f[2 * e + 1]) : 0.f) + (s1 >= lane ? as_f(b[2 * e + 1]) : 0.f);
+                pk[8 * h + e] = pack_bf16(lo, hi);
+            }
+        }
+    }
+}
+__device__ __forceinline__ void combine_any(int cb, int wq, bool valid, uint32_t fwd_addr, uint32_t bwd_addr, int lane,
+                                            uint32_t (&pk)[16]) {
+    if (!valid) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) pk[e] = 0u;
+    } else if (cb < wq) {
+        combine_block<-1>(fwd_addr, bwd_addr, lane, pk);
+    } else if (cb == wq) {
+        combine_block<0>(fwd_addr, bwd_addr, lane, pk);
+    } else {
+        combine_block<1>(fwd_addr, bwd_addr, lane, pk);
+    }
+}
+
+// Shared-memory matrix descriptor, in halves.  Low word: start address and leading-dimension byte
+// offset, both in 16-byte units (bits 0..13 and 16..29), so stepping an operand through shared memory is
+// one 32-bit add.  High word: stride-dimension byte offset in 16-byte units (bits 32..45), descriptor
+// version 1 (bit 46), swizzle mode in bits 61..63 (0 = none, 2 = 128B, 4 = 64B).
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+    return ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes, uint32_t swizzle) {
+    return (sbo_bytes >> 4) | (1u << 14) | (swizzle << 29);
+}
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) { return ((uint64_t)hi << 32) | lo; }
+
+constexpr uint32_t kHiK64 = desc_hi(512, 4);     // K-major or MN-major tile with 64-byte rows, 64B swizzle
+constexpr uint32_t kHiV128 = desc_hi(1024, 2);   // MN-major tile with 128-byte rows, 128B swizzle
+constexpr uint32_t kHiZ = desc_hi(256, 0);       // 0/1 tiles, no swizzle
+
+// 1 / x for a normal, positive x without the special-function unit: a bit-level first guess (within 5.1 %)
+// and Newton steps (one: relative error below 0.26 %, two: below 1e-5).  The result only scales bf16
+// operands (rounding unit 0.39 %).
+template <int STEPS>
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r = __uint_as_float(0x7EF311C7u - __float_as_uint(x));
+#pragma unroll
+    for (int i = 0; i < STEPS; ++i) r = r * fmaf(-x, r, 2.0f);
+    return r;
+}
+constexpr int kRcpSteps = 2;
+
+// Builds the two 240-row 0/1 tiles of the prefix / suffix sums (K-major without swizzle: 8-row groups of 256
+// bytes, each two 8x8 core matrices for K 0..7 and K 8..15).  Rows 0..111 of `zf` are zeros, rows 112..127 the
+// lower triangle (diagonal included), rows 128..239 ones; `zb` holds ones, the upper triangle, zeros.  The
+// 128-row window starting at row 112 - 16 j is the operand of K step j.  Threads 0..239 of the block write.
+__device__ __forceinline__ void build_zero_one_tiles(uint8_t* zf, uint8_t* zb, int tid) {
+    if (tid < (int)kZRows) {
+        uint32_t f[8], b[8];
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            uint32_t wf = 0, wb = 0;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int kk = 2 * p + h, u = tid - 112;
+                const bool one_f = tid >= 128 || (tid >= 112 && kk <= u);
+                const bool one_b = tid < 112 || (tid < 128 && kk >= u);
+                wf |= (one_f ? 0x3F80u : 0u) << (16 * h);
+                wb |= (one_b ? 0x3F80u : 0u) << (16 * h);
+            }
+            f[p] = wf;
+            b[p] = wb;
+        }
+        const uint32_t off = (uint32_t)(tid >> 3) * 256 + (uint32_t)(tid & 7) * 16;
+        *reinterpret_cast<uint4*>(zf + off) = make_uint4(f[0], f[1], f[2], f[3]);
+        *reinterpret_cast<uint4*>(zf + off + 128) = make_uint4(f[4], f[5], f[6], f[7]);
+        *reinterpret_cast<uint4*>(zb + off) = make_uint4(b[0], b[1], b[2], b[3]);
+        *reinterpret_cast<uint4*>(zb + off + 128) = make_uint4(b[4], b[5], b[6], b[7]);
+    }
+}
+
+}  // namespace umma
+}  // namespace vig

@@ -39,6 +39,12 @@ cudaError_t launch_bigla_umma(const __nv_bfloat16* q, const __nv_bfloat16* k, co
                               const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
                               long long units, int L, int dk, int dv, cudaStream_t stream);
 
+// ---- bf16 tcgen05 / TMEM path for longer sequences: chunk tasks, states through scratch (three launches) ----
+size_t umma_long_workspace_bytes(long long units, int L, int dk, int dv);
+cudaError_t launch_bigla_umma_long(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                   const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
+                                   long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
+
 // Kernel family the bf16 entry points prefer (VIG_KERNEL_*), set by vig_set_kernel_preference.
 int kernel_preference();
 
