@@ -22,6 +22,8 @@
 // two blocks share an SM and one block's MMA round trips hide behind the other's element-wise phases.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "ptx.cuh"
 #include "recurrence.cuh"
 #include "tma_host.h"
@@ -36,6 +38,7 @@ using namespace umma;
 constexpr int kMaxRows = 256;   // longest unit this kernel takes
 constexpr int kThreads = 256;
 constexpr uint32_t kTmemCols = 256;
+constexpr int kMaxDevices = 64;
 
 // ---- shared-memory plan (rows = tokens of the unit rounded up to 16) ---------------------------
 struct ULayout {
@@ -521,16 +524,24 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows; a.units = units;
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return cudaErrorUnknown;
     // The MMAs of chunk 1 read 128 rows of the operand tiles from row 128 on, i.e. up to (256 - rows) * 64
     // bytes past the last q-type tile: that lands in the v tile, inside the allocation.
     size_t smem = make_layout(rows).total + 1024;   // slack for the manual 1 KB alignment
     const size_t rec = (size_t)rec_plan(kThreads, DK, DV).smem_floats * 4 + 1024;
     if (smem < rec) smem = rec;
-    cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    // once per device: shared-memory opt-in (for the longest unit the kernel takes) and the SM count
+    static std::atomic<int> sms_of[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int sms = sms_of[dev].load(std::memory_order_acquire);
+    if (sms == 0) {
+        size_t most = make_layout(kMaxRows).total + 1024;
+        if (most < rec) most = rec;
+        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+        if (e != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        sms_of[dev].store(sms, std::memory_order_release);
+    }
     // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...
     const long long grid = units < 2LL * sms ? units : 2LL * sms;
     bigla_umma_kernel<DK, DV><<<(unsigned)grid, kThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);

@@ -13,6 +13,8 @@
 // owns token r of the chunk in every element-wise phase.  All products are tcgen05.mma with M = 128.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "recurrence.cuh"
 #include "tma_host.h"
 #include "umma.cuh"
@@ -26,13 +28,15 @@ using namespace umma;
 constexpr int kLThreads = 128;
 constexpr uint32_t kLTmemCols = 128;
 constexpr int kLBlocksPerSm = 3;
+constexpr int kMaxDevices = 64;
 enum LongMode { kLMain = 0, kLSummary = 1 };
 
 // ---- scratch ---------------------------------------------------------------------------------------------
 // slot(unit, chunk, dir): 32 x DV fp32 (summary, key dim major), overwritten by the fold with a 4 KB bf16 tile
-// image [32][64] (128-byte rows, 128B swizzle);  decay(unit, chunk, dir): 32 fp32;  flags(unit): int.
+// image [32][64] (128-byte rows, 128B swizzle);  decay(unit, chunk, dir): 32 fp32;  flags(unit), chunk flags(unit, chunk): int.
+// Every word is written before it is read within one call: nothing has to be cleared beforehand.
 struct LongWs {
-    size_t slot_bytes, decay_off, flags_off, total;
+    size_t slot_bytes, decay_off, flags_off, cflags_off, total;
 };
 LongWs long_ws_layout(long long units, int nch, int dv) {
     LongWs w;
@@ -40,7 +44,8 @@ LongWs long_ws_layout(long long units, int nch, int dv) {
     w.slot_bytes = (size_t)32 * dv * 4 < 4096 ? 4096 : (size_t)32 * dv * 4;
     w.decay_off = up((size_t)units * nch * 2 * w.slot_bytes);
     w.flags_off = w.decay_off + up((size_t)units * nch * 2 * 32 * 4);
-    w.total = w.flags_off + up((size_t)units * 4);
+    w.cflags_off = w.flags_off + up((size_t)units * 4);
+    w.total = w.cflags_off + up((size_t)units * nch * 4);
     return w;
 }
 
@@ -64,7 +69,8 @@ struct LArgs {
     long long tasks;
     uint8_t* ws_slots;    // [units][nch][2][slot_bytes]
     float* ws_decay;      // [units][nch][2][32]
-    int* ws_flags;        // [units]
+    int* ws_flags;        // [units]: the unit needs the exact recurrence (written by the fold launch)
+    int* ws_cflags;       // [units][nch]: per-chunk range check of the summary launch
     uint32_t slot_bytes;
     int* dev_status;
 };
@@ -338,7 +344,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 args.ws_decay[((size_t)task * 2 + dir) * 32 + lane] = d;
             }
             handover();
-            if (tid == 0 && (slow_slot[0] | slow_slot[1]) != 0) args.ws_flags[unit] = 1;
+            if (tid == 0) args.ws_cflags[task] = slow_slot[0] | slow_slot[1];
             if (*time_flag != 0) break;
             if (ctl && has_next) {
                 load_operands(next);
@@ -489,24 +495,29 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 }
 
 // Sequential fold of the chunk summaries of one unit and direction.  Thread (i, c) owns the eight value dims
-// 8 c .. 8 c + 7 of key dim i.  Chunks are taken in batches of eight so that their loads are all in flight
+// 8 c .. 8 c + 7 of key dim i.  Chunks are taken in batches of sixteen so that their loads are all in flight
 // together; after a batch is in registers the incoming states are written, as bf16 tile images, over the
-// first 4 KB of the same slots.
+// first 4 KB of the same slots.  The block also reduces the chunks' range flags to the unit's flag.
 template <int DV>
 __global__ void __launch_bounds__(32 * (DV / 8))
-bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, const int* ws_flags, int nch, uint32_t slot_bytes) {
+bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, int* ws_flags, const int* ws_cflags, int nch, uint32_t slot_bytes) {
     constexpr int CPR = DV / 8;   // 16-byte chunks of live value dims per row of the image
+    constexpr int kBatch = 16;
     const int unit = blockIdx.x, dir = blockIdx.y;
-    if (ws_flags[unit] != 0) return;
+    int flagged = 0;
+    for (int m = threadIdx.x; m < nch; m += blockDim.x) flagged |= ws_cflags[(size_t)unit * nch + m];
+    flagged = __syncthreads_or(flagged);
+    if (dir == 0 && threadIdx.x == 0) ws_flags[unit] = flagged;
+    if (flagged) return;   // the main launch redoes the unit by the recurrence
     const int i = threadIdx.x / CPR, c = threadIdx.x % CPR;
     float carry[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) carry[e] = 0.f;
-    for (int mb = 0; mb < nch; mb += 8) {
-        float4 u[8][2];
-        float d[8];
+    for (int mb = 0; mb < nch; mb += kBatch) {
+        float4 u[kBatch][2];
+        float d[kBatch];
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
+        for (int b = 0; b < kBatch; ++b) {
             if (mb + b < nch) {
                 const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
                 const size_t s = ((size_t)unit * nch + m) * 2 + dir;
@@ -518,7 +529,7 @@ bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, const int* ws_f
         }
         __syncthreads();   // every summary of the batch is in registers before any of its slots is overwritten
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
+        for (int b = 0; b < kBatch; ++b) {
             if (mb + b < nch) {
                 const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
                 uint8_t* img = ws_slots + (((size_t)unit * nch + m) * 2 + dir) * slot_bytes;
@@ -533,7 +544,6 @@ bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, const int* ws_f
                 for (int e = 0; e < 8; ++e) carry[e] = fmaf(carry[e], d[b], uu[e]);
             }
         }
-        __syncthreads();   // images written before the next batch's loads (they touch other slots, but keep the order plain)
     }
 }
 
@@ -554,23 +564,29 @@ cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     a.ws_slots = static_cast<uint8_t*>(ws);
     a.ws_decay = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + wl.decay_off);
     a.ws_flags = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + wl.flags_off);
+    a.ws_cflags = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + wl.cflags_off);
     a.slot_bytes = (uint32_t)wl.slot_bytes;
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return cudaErrorUnknown;
     size_t smem = LLayout::total + 1024;   // slack for the manual 1 KB alignment
     const size_t rec = (size_t)rec_plan(kLThreads, DK, DV).smem_floats * 4 + 1024;
     if (smem < rec) smem = rec;
-    cudaError_t e;
-    if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLSummary>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLMain>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(a.ws_flags, 0, (size_t)units * 4, stream)) != cudaSuccess) return e;
+    // once per device: shared-memory opt-in of the two kernels and the SM count
+    static std::atomic<int> sms_of[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int sms = sms_of[dev].load(std::memory_order_acquire);
+    if (sms == 0) {
+        cudaError_t e;
+        if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLSummary>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLMain>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        sms_of[dev].store(sms, std::memory_order_release);
+    }
     const long long cap = (long long)kLBlocksPerSm * sms;
     const unsigned grid = (unsigned)(a.tasks < cap ? a.tasks : cap);   // persistent blocks: block b takes tasks b, b + grid, ...
     bigla_long_kernel<DK, DV, kLSummary><<<grid, kLThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
-    bigla_long_fold_kernel<DV><<<dim3((unsigned)units, 2), 32 * (DV / 8), 0, stream>>>(a.ws_slots, a.ws_decay, a.ws_flags, nch, a.slot_bytes);
+    bigla_long_fold_kernel<DV><<<dim3((unsigned)units, 2), 32 * (DV / 8), 0, stream>>>(a.ws_slots, a.ws_decay, a.ws_flags, a.ws_cflags, nch, a.slot_bytes);
     bigla_long_kernel<DK, DV, kLMain><<<grid, kLThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
     count_launch(3);
     return cudaGetLastError();

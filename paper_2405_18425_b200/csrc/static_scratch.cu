@@ -56,8 +56,8 @@ extern "C" int vig_bigla_fwd_static_bf16(const void* q, const void* k, const voi
     if (B == 0 || H == 0 || L == 0) return VIG_OK;
     void* scratch = nullptr;
     if (static_scratch_ptr(&scratch) != cudaSuccess) return VIG_ERR_CUDA;
-    // The launcher clears the per-unit flags inside the scratch with a memset on `stream` before the
-    // first kernel; everything else in it is written before it is read within the same call.
+    // Nothing in the scratch has to survive from call to call: the launcher clears the words that must start at
+    // zero on `stream`, and everything else in it is written before it is read within the same call.
     cudaError_t e = launch_bigla_mma((const bf*)q, (const bf*)k, (const bf*)v, (const bf*)log_alpha_fwd,
                                      (const bf*)log_alpha_bwd, (bf*)out, units, L, dk, dv, scratch,
                                      (cudaStream_t)stream);
