@@ -127,6 +127,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tma_load_3d(t_v, &tm_v, 0, 0, unit, bar_v);
     };
 
+    pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
     if (tid == 0) {
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
@@ -135,9 +136,6 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
         for (int i = 0; i < 4; ++i) slow_slot[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        // the first loads go out at once: the rest of the set-up overlaps their latency
-        load_gates_qk(blockIdx.x);
-        load_v(blockIdx.x);
     }
     __syncwarp();
     if (warp == 0) {
@@ -145,6 +143,11 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     build_zero_one_tiles(bp + lay.zf, bp + lay.zb, tid);
+    pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
+    if (tid == 0) {
+        load_gates_qk(blockIdx.x);
+        load_v(blockIdx.x);
+    }
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -544,9 +547,9 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     }
     // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...
     const long long grid = units < 2LL * sms ? units : 2LL * sms;
-    bigla_umma_kernel<DK, DV><<<(unsigned)grid, kThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
+    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
     count_launch();
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 }  // namespace

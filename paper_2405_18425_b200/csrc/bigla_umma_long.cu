@@ -132,6 +132,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tma_load_3d(t_v, &tm_v, 0, task_chunk(t) * kChunk, task_unit(t), bar_v);
     };
 
+    pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
     if (tid == 0) {
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
@@ -147,6 +148,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // the 240 rows of the 0/1 tiles, two passes of 128 threads
     build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid);
     build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid + kLThreads);
+    pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     fence_async_smem();
     tc_fence_before();
     __syncthreads();
@@ -504,6 +506,8 @@ bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, int* ws_flags, 
     constexpr int CPR = DV / 8;   // 16-byte chunks of live value dims per row of the image
     constexpr int kBatch = 16;
     const int unit = blockIdx.x, dir = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();
     int flagged = 0;
     for (int m = threadIdx.x; m < nch; m += blockDim.x) flagged |= ws_cflags[(size_t)unit * nch + m];
     flagged = __syncthreads_or(flagged);
@@ -585,9 +589,13 @@ cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     }
     const long long cap = (long long)kLBlocksPerSm * sms;
     const unsigned grid = (unsigned)(a.tasks < cap ? a.tasks : cap);   // persistent blocks: block b takes tasks b, b + grid, ...
-    bigla_long_kernel<DK, DV, kLSummary><<<grid, kLThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
-    bigla_long_fold_kernel<DV><<<dim3((unsigned)units, 2), 32 * (DV / 8), 0, stream>>>(a.ws_slots, a.ws_decay, a.ws_flags, a.ws_cflags, nch, a.slot_bytes);
-    bigla_long_kernel<DK, DV, kLMain><<<grid, kLThreads, smem, stream>>>(tq, tk, tf, tb, tv, to, a);
+    cudaError_t le = launch_pdl(bigla_long_kernel<DK, DV, kLSummary>, dim3(grid), dim3(kLThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    if (le == cudaSuccess)
+        le = launch_pdl(bigla_long_fold_kernel<DV>, dim3((unsigned)units, 2), dim3(32 * (DV / 8)), 0, stream, a.ws_slots,
+                        (const float*)a.ws_decay, a.ws_flags, (const int*)a.ws_cflags, nch, a.slot_bytes);
+    if (le == cudaSuccess)
+        le = launch_pdl(bigla_long_kernel<DK, DV, kLMain>, dim3(grid), dim3(kLThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    if (le != cudaSuccess) return le;
     count_launch(3);
     return cudaGetLastError();
 }

@@ -1,4 +1,5 @@
 // Gate preparation: log alpha = logsigmoid(g) / tau (paper Eq. 5 line 1), both directions in one launch.
+#include "ptx.cuh"
 #include "vig_internal.h"
 
 namespace vig {
@@ -36,6 +37,8 @@ __device__ __forceinline__ uint4 log_alpha_bf16x8(uint4 raw, float inv_tau) {
 template <typename T>
 __global__ void __launch_bounds__(256) gate_prep_kernel(const T* g_f, const T* g_b, T* la_f, T* la_b, long long n, float inv_tau) {
     // no __restrict__: the output may alias the input (in-place call)
+    pdl_launch_dependents();
+    pdl_wait();
     const T* g = blockIdx.y == 0 ? g_f : g_b;
     T* la = blockIdx.y == 0 ? la_f : la_b;
     constexpr int V = 16 / sizeof(T);
@@ -75,9 +78,9 @@ cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long 
     long long blocks = (n / V + threads - 1) / threads;
     if (blocks < 1) blocks = 1;
     if (blocks > 148 * 4) blocks = 148 * 4;   // both directions together: eight blocks per SM
-    gate_prep_kernel<T><<<dim3((unsigned)blocks, 2), threads, 0, stream>>>(g_f, g_b, la_f, la_b, n, 1.0f / tau);
+    const cudaError_t le = launch_pdl(gate_prep_kernel<T>, dim3((unsigned)blocks, 2), dim3(threads), 0, stream, g_f, g_b, la_f, la_b, n, 1.0f / tau);
     count_launch();
-    return cudaGetLastError();
+    return le != cudaSuccess ? le : cudaGetLastError();
 }
 
 template cudaError_t launch_gate_prep<float>(const float*, const float*, float*, float*, long long, float,

@@ -94,6 +94,13 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
+// Programmatic dependent launch.  `pdl_launch_dependents`: the next kernel in the stream, if it was launched with
+// programmatic stream serialization, may start its prologue once every block of this grid has executed this (or
+// exited).  `pdl_wait`: blocks until every kernel this grid depends on has completed and its memory operations are
+// visible; a no-op for an ordinary launch.  The kernels here execute it before their first global-memory access.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Byte offset of 16-byte chunk `chunk` of row `row` in a TMA-swizzled tile whose rows are RB bytes
 // (RB = 32, 64 or 128 = the swizzle span; tile base aligned to 8 rows of the span).
 template <int RB>

@@ -141,7 +141,7 @@ __device__ __forceinline__ float fast_rcp(float x) {
     for (int i = 0; i < STEPS; ++i) r = r * fmaf(-x, r, 2.0f);
     return r;
 }
-constexpr int kRcpSteps = 2;
+constexpr int kRcpSteps = 1;
 
 // Builds the two 240-row 0/1 tiles of the prefix / suffix sums (K-major without swizzle: 8-row groups of 256
 // bytes, each two 8x8 core matrices for K 0..7 and K 8..15).  Rows 0..111 of `zf` are zeros, rows 112..127 the

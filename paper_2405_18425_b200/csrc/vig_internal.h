@@ -45,6 +45,24 @@ cudaError_t launch_bigla_umma_long(const __nv_bfloat16* q, const __nv_bfloat16* 
                                    const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
                                    long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
 
+// Launch with programmatic stream serialization: the kernel's prologue (everything before its pdl_wait) may overlap
+// the tail of the kernel before it in the stream.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Kernel family the bf16 entry points prefer (VIG_KERNEL_*), set by vig_set_kernel_preference.
 int kernel_preference();
 
