@@ -48,7 +48,7 @@ struct ULayout {
     uint32_t zf, zb;   // 0/1 tiles of the prefix / suffix sums
     uint32_t s_fwd;    // bf16 state entering chunk 1 from the left  [32][64] (128B swizzle)
     uint32_t s_bwd;    // bf16 state entering chunk 0 from the right
-    uint32_t dec;      // [2][32] fp32 chunk totals of the log gates: b at the last row of chunk 0, e at the first row of chunk 1
+    uint32_t dec;      // [2 chunks][2][32] fp32 totals of the log gates: b at the chunk's last row, e at its first row
     uint32_t misc;     // six mbarriers, TMEM slot, flags
     uint32_t total;
 };
@@ -61,7 +61,7 @@ __host__ __device__ inline ULayout make_layout(int rows) {
     l.s_fwd = (l.zb + kZBytes + 1023u) & ~1023u;
     l.s_bwd = l.s_fwd + 32 * 128;
     l.dec = l.s_bwd + 32 * 128;
-    l.misc = l.dec + 2 * 32 * 4;
+    l.misc = l.dec + 4 * 32 * 4;
     l.total = l.misc + 128;
     return l;
 }
@@ -104,7 +104,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_pfx = bar_g + 40, slot = bar_g + 48;
     volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 48);
     volatile int* time_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 52);
-    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 56);   // [4]: (chunk, first / last row) range checks
+    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 56);   // [4]: range check per chunk (two used)
     const int ks_c1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;                          // K steps of chunk 1
     const int npass_c1 = ks_c1 > 4 ? 2 : 1;
     const int ks_c0 = (min(L, kChunk) + 15) >> 4;                                     // K steps of chunk 0
@@ -143,6 +143,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     build_zero_one_tiles(bp + lay.zf, bp + lay.zb, tid);
+    if (tid < 128) dec[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     if (tid == 0) {
         load_gates_qk(blockIdx.x);
@@ -224,7 +225,6 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 constexpr int kHalves = (DK + 15) / 16;
                 const int last_row = min(L, (c + 1) * kChunk) - 1;
                 const bool check_row = row_live && (row == last_row || row == c * kChunk);
-                float mfa = 0.f, mba = 0.f;
                 uint32_t pf[kHalves][16], pb[kHalves][16];
                 tmem_ld16(rl + 32 * c, pf[0]);
                 tmem_ld16(rl + 64 + 32 * c, pb[0]);
@@ -241,20 +241,17 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         asm volatile("bar.arrive 3, 256;" ::: "memory");
                     }
                     if (check_row) {
-                        // b is smallest at the last row of the chunk, e at its first row (tree minima: these two
-                        // threads hold their whole warps up)
-                        float mf[4] = {0.f, 0.f, 0.f, 0.f}, mb[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                        for (int d = 0; d < 16; ++d) { mf[d & 3] = fminf(mf[d & 3], as_f(pf[hf][d])); mb[d & 3] = fminf(mb[d & 3], as_f(pb[hf][d])); }
-                        mfa = fminf(mfa, fminf(fminf(mf[0], mf[1]), fminf(mf[2], mf[3])));
-                        mba = fminf(mba, fminf(fminf(mb[0], mb[1]), fminf(mb[2], mb[3])));
-                        // chunk totals of the log gates for the state hand-over: b at the last row of chunk 0, e at the first row of chunk 1
-                        if (nc == 2 && (row == kChunk - 1 || row == kChunk)) {
-                            uint4* dst = reinterpret_cast<uint4*>(dec + (row == kChunk ? 32 : 0) + 16 * hf);
+                        // totals of the log gates over the chunk: b at its last row, e at its first row.  They feed the
+                        // range check (done by a whole warp after the hand-over) and the decay of the chunk summaries.
+                        if (row == last_row) {
 #pragma unroll
                             for (int x = 0; x < 4; ++x)
-                                dst[x] = row == kChunk ? make_uint4(pb[hf][4 * x], pb[hf][4 * x + 1], pb[hf][4 * x + 2], pb[hf][4 * x + 3])
-                                                       : make_uint4(pf[hf][4 * x], pf[hf][4 * x + 1], pf[hf][4 * x + 2], pf[hf][4 * x + 3]);
+                                reinterpret_cast<uint4*>(dec + (2 * c) * 32 + 16 * hf)[x] = make_uint4(pf[hf][4 * x], pf[hf][4 * x + 1], pf[hf][4 * x + 2], pf[hf][4 * x + 3]);
+                        }
+                        if (row == c * kChunk) {
+#pragma unroll
+                            for (int x = 0; x < 4; ++x)
+                                reinterpret_cast<uint4*>(dec + (2 * c + 1) * 32 + 16 * hf)[x] = make_uint4(pb[hf][4 * x], pb[hf][4 * x + 1], pb[hf][4 * x + 2], pb[hf][4 * x + 3]);
                         }
                     }
                     if (row_live) {
@@ -285,10 +282,6 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         }
                     }
                 }
-                if (check_row) {
-                    if (row == last_row) slow_slot[2 * c + 1] = mfa < -kGateRange ? 1 : 0;
-                    if (row == c * kChunk) slow_slot[2 * c] = mba < -kGateRange ? 1 : 0;
-                }
             }
             if (c == 1 && !warp_live) {   // warps of chunk 1 without tokens read no sums but still take part in the hand-over
                 asm volatile("bar.arrive 3, 256;" ::: "memory");
@@ -301,6 +294,12 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_fence_after();
             } else {
                 chunk_handover();
+            }
+            if (wq == 2) {
+                // range check, one key dim per lane: b is smallest at the last row of the chunk, e at its first row
+                const bool out_of_range = dec[(2 * c) * 32 + lane] < -kGateRange || dec[(2 * c + 1) * 32 + lane] < -kGateRange;
+                const bool any = __any_sync(0xffffffffu, out_of_range);
+                if (lane == 0) slow_slot[c] = any ? 1 : 0;
             }
             if (ctl && v_load_pending) {
                 // The store of the previous unit was issued a phase ago and has read the v tile by now: this
@@ -382,7 +381,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (warp == 1 || warp == 4) {
                     // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
                     // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
-                    const float d = ex2(dec[(warp == 1 ? 0 : 32) + lane] * kLog2e);   // decay of the whole chunk for key dim `lane`
+                    const float d = ex2(dec[(warp == 1 ? 0 : 96) + lane] * kLog2e);   // decay of the whole chunk for key dim `lane`
                     uint8_t* st = bp + (warp == 1 ? lay.s_fwd : lay.s_bwd);
 #pragma unroll
                     for (int hb = 0; hb < 2; ++hb) {

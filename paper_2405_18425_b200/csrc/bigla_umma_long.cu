@@ -59,7 +59,7 @@ struct LLayout {
     static constexpr uint32_t s_fwd = (zb + kZBytes + 1023u) & ~1023u;   // incoming states, bf16 [32][64], 128B swizzle
     static constexpr uint32_t s_bwd = s_fwd + 4096;
     static constexpr uint32_t misc = s_bwd + 4096;     // mbarriers, TMEM slot, flags
-    static constexpr uint32_t total = misc + 128;
+    static constexpr uint32_t total = misc + 64 + 256;
 };
 
 struct LArgs {
@@ -100,8 +100,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t slot = bar_g + 40;
     volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + Y::misc + 40);
     volatile int* time_flag = reinterpret_cast<volatile int*>(bp + Y::misc + 44);
-    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + Y::misc + 48);   // [2]: first-row / last-row range checks
-    float* totals = reinterpret_cast<float*>(bp + Y::s_fwd);   // summary mode: [2][32] chunk totals of the log gates (state tiles unused there)
+    volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + Y::misc + 48);   // range check of the chunk (summary mode)
+    float* totals = reinterpret_cast<float*>(bp + Y::misc + 64);   // [2][32] chunk totals of the log gates: b at the last row, e at the first row
     uint32_t mma_phase = 0;
 
     const uint32_t t_kb = base, t_kf = base + Y::tile, t_qf = base + 2 * Y::tile, t_qb = base + 3 * Y::tile;
@@ -137,7 +137,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
         *time_flag = 0;
-        slow_slot[0] = slow_slot[1] = 0;
+        slow_slot[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (wq == 0) {
@@ -148,6 +148,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // the 240 rows of the 0/1 tiles, two passes of 128 threads
     build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid);
     build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid + kLThreads);
+    if (tid < 64) totals[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     fence_async_smem();
     tc_fence_before();
@@ -221,7 +222,6 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (warp_live) {
             constexpr int kHalves = (DK + 15) / 16;
             const bool check_row = row_live && (row == rows_here - 1 || row == 0);
-            float mfa = 0.f, mba = 0.f;
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) {
                 uint32_t pf[16], pb[16];
@@ -229,24 +229,17 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tmem_ld16(rc + 32 + 16 * hf, pb);
                 tc_wait_ld();
                 if (check_row) {
-                    // b is smallest at the last row of the chunk, e at its first row
-                    float mf[4] = {0.f, 0.f, 0.f, 0.f}, mb[4] = {0.f, 0.f, 0.f, 0.f};
+                    // totals of the log gates over the chunk: b at its last row, e at its first row (range check after
+                    // the hand-over, decay of the summary)
+                    if (row == rows_here - 1) {
 #pragma unroll
-                    for (int d = 0; d < 16; ++d) { mf[d & 3] = fminf(mf[d & 3], as_f(pf[d])); mb[d & 3] = fminf(mb[d & 3], as_f(pb[d])); }
-                    mfa = fminf(mfa, fminf(fminf(mf[0], mf[1]), fminf(mf[2], mf[3])));
-                    mba = fminf(mba, fminf(fminf(mb[0], mb[1]), fminf(mb[2], mb[3])));
-                    if (MODE == kLSummary) {
-                        // chunk totals of the log gates: b at the last row, e at the first row
-                        if (row == rows_here - 1) {
+                        for (int x = 0; x < 4; ++x)
+                            reinterpret_cast<uint4*>(totals + 16 * hf)[x] = make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
+                    }
+                    if (row == 0) {
 #pragma unroll
-                            for (int x = 0; x < 4; ++x)
-                                reinterpret_cast<uint4*>(totals + 16 * hf)[x] = make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
-                        }
-                        if (row == 0) {
-#pragma unroll
-                            for (int x = 0; x < 4; ++x)
-                                reinterpret_cast<uint4*>(totals + 32 + 16 * hf)[x] = make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3]);
-                        }
+                        for (int x = 0; x < 4; ++x)
+                            reinterpret_cast<uint4*>(totals + 32 + 16 * hf)[x] = make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3]);
                     }
                 }
                 if (row_live) {
@@ -296,16 +289,18 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         if (!row_live || ch >= DK / 8) *reinterpret_cast<uint4*>(bp + sw_off<64>(row, ch)) = make_uint4(0, 0, 0, 0);
                 }
             }
-            if (check_row) {
-                if (row == rows_here - 1) slow_slot[1] = mfa < -kGateRange ? 1 : 0;
-                if (row == 0) slow_slot[0] = mba < -kGateRange ? 1 : 0;
-            }
         } else if (MODE == kLSummary) {
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) *reinterpret_cast<uint4*>(bp + sw_off<64>(row, ch)) = make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
         handover();
+        if (wq == 2 && MODE == kLSummary) {
+            // range check, one key dim per lane: b is smallest at the last row of the chunk, e at its first row
+            const bool out_of_range = totals[lane] < -kGateRange || totals[32 + lane] < -kGateRange;
+            const bool any = __any_sync(0xffffffffu, out_of_range);
+            if (lane == 0) slow_slot[0] = any ? 1 : 0;
+        }
         if (ctl && v_load_pending) {
             // the store of the previous task has read the v tile by now; the tile is needed again only further down
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
@@ -328,7 +323,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (wq < 2) {
                 // lane = key dim; warp 0: backward summary, warp 1: forward summary
                 const int dir = wq == 1 ? 0 : 1;
-                const float d = lane < DK ? ex2(totals[(dir == 0 ? 0 : 32) + lane] * kLog2e) : 1.f;   // decay of the whole chunk for this key dim
+                const float d = ex2(totals[(dir == 0 ? 0 : 32) + lane] * kLog2e);   // decay of the whole chunk for this key dim
                 float* dst = reinterpret_cast<float*>(args.ws_slots + ((size_t)task * 2 + dir) * args.slot_bytes) + (size_t)lane * DV;
 #pragma unroll
                 for (int hb = 0; hb < 2; ++hb) {
@@ -346,7 +341,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 args.ws_decay[((size_t)task * 2 + dir) * 32 + lane] = d;
             }
             handover();
-            if (tid == 0) args.ws_cflags[task] = slow_slot[0] | slow_slot[1];
+            if (tid == 0) args.ws_cflags[task] = slow_slot[0];
             if (*time_flag != 0) break;
             if (ctl && has_next) {
                 load_operands(next);
