@@ -205,6 +205,7 @@ int vig_last_device_status(void* stream) {
         const int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return VIG_ERR_CUDA;
     }
+    if (word & kDevStatusInternal) return VIG_ERR_CUDA;
     return (word & kDevStatusTimeout) ? VIG_ERR_DEVICE_TIMEOUT : VIG_OK;
 }
 

@@ -27,7 +27,8 @@ using namespace umma;
 
 constexpr int kLThreads = 128;
 constexpr uint32_t kLTmemCols = 128;
-constexpr int kLBlocksPerSm = 3;
+constexpr int kLBlocksPerSm = 3;          // main launch: blocks per SM (shared memory)
+constexpr int kLSummaryBlocksPerSm = 4;   // summary launch (shared memory and TMEM: 4 x 128 columns)
 constexpr int kMaxDevices = 64;
 enum LongMode { kLMain = 0, kLSummary = 1 };
 
@@ -50,15 +51,24 @@ LongWs long_ws_layout(long long units, int nch, int dv) {
 }
 
 // ---- shared memory -------------------------------------------------------------------------------------------
+// Main mode holds four q-type tiles [128][32] bf16 (64B swizzle; loaded: q, k, log alpha>, log alpha<; scaled in
+// place: k~<, k~>, q~>, q~<), the v tile (later the output tile), the 0/1 tiles and the two incoming states.
+// Summary mode needs neither q nor states and writes k~< over the log alpha> tile once the prefix sums are taken,
+// which keeps a block below a quarter of an SM's shared memory.
+template <int MODE>
 struct LLayout {
-    static constexpr uint32_t tile = 128 * 64;         // q-type tile [128][32] bf16, 64B swizzle; four from offset 0:
-                                                       //   loaded: q, k, log alpha>, log alpha<; scaled: k~<, k~>, q~>, q~<
-    static constexpr uint32_t v = 4 * tile;            // v tile [128][64] bf16 (128B swizzle), later the output tile
+    static constexpr uint32_t tile = 128 * 64;
+    static constexpr uint32_t k = MODE == kLMain ? tile : 0;             // k, then k~>
+    static constexpr uint32_t f = k + tile;                               // log alpha>, then q~> (main) / k~< (summary)
+    static constexpr uint32_t b = f + tile;                               // log alpha<, then q~< (main)
+    static constexpr uint32_t q = 0;                                      // main only: q, then k~<
+    static constexpr uint32_t kb = MODE == kLMain ? q : f;                // where k~< lives
+    static constexpr uint32_t v = b + tile;                               // v tile [128][64] bf16 (128B swizzle)
     static constexpr uint32_t zf = v + 128 * 128;
     static constexpr uint32_t zb = zf + kZBytes;
-    static constexpr uint32_t s_fwd = (zb + kZBytes + 1023u) & ~1023u;   // incoming states, bf16 [32][64], 128B swizzle
+    static constexpr uint32_t s_fwd = (zb + kZBytes + 1023u) & ~1023u;    // main only: incoming states, bf16 [32][64], 128B swizzle
     static constexpr uint32_t s_bwd = s_fwd + 4096;
-    static constexpr uint32_t misc = s_bwd + 4096;     // mbarriers, TMEM slot, flags
+    static constexpr uint32_t misc = MODE == kLMain ? s_bwd + 4096 : zb + kZBytes;   // mbarriers, TMEM slot, flags, totals
     static constexpr uint32_t total = misc + 64 + 256;
 };
 
@@ -82,15 +92,19 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
 }
 
 template <int DK, int DV, int MODE>
-__global__ void __launch_bounds__(kLThreads, kLBlocksPerSm)
+__global__ void __launch_bounds__(kLThreads, MODE == kLSummary ? kLSummaryBlocksPerSm : kLBlocksPerSm)
 bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const LArgs args) {
     static_assert((DK == 16 || DK == 24 || DK == 32) && (DV == 32 || DV == 48 || DV == 64), "unsupported head size");
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* bp = smem_raw + (base - smem_u32(smem_raw));
-    using Y = LLayout;
+    extern __shared__ __align__(1024) uint8_t smem_raw[];   // the swizzled tiles need the 1 KB alignment; no slack is allocated
+    const uint32_t base = smem_u32(smem_raw);
+    uint8_t* bp = smem_raw;
+    using Y = LLayout<MODE>;
+    if ((base & 1023u) != 0) {   // never expected: reported instead of computing on misplaced tiles
+        if (threadIdx.x == 0) atomicOr(args.dev_status, kDevStatusInternal);
+        return;
+    }
 
     const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
     const int L = args.L, nch = args.nch;
@@ -104,7 +118,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     float* totals = reinterpret_cast<float*>(bp + Y::misc + 64);   // [2][32] chunk totals of the log gates: b at the last row, e at the first row
     uint32_t mma_phase = 0;
 
-    const uint32_t t_kb = base, t_kf = base + Y::tile, t_qf = base + 2 * Y::tile, t_qb = base + 3 * Y::tile;
+    const uint32_t t_kb = base + Y::kb, t_kf = base + Y::k, t_qf = base + Y::f, t_qb = base + Y::b, t_q = base + Y::q;
     const uint32_t t_v = base + Y::v;
 
     auto task_unit = [&](long long t) { return (int)(t / nch); };
@@ -116,7 +130,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tma_load_3d(t_qb, &tm_b, 0, r0, u, bar_g);
         if (MODE == kLMain) {
             mbar_expect_tx(bar_qk, 2 * Y::tile);
-            tma_load_3d(t_kb, &tm_q, 0, r0, u, bar_qk);
+            tma_load_3d(t_q, &tm_q, 0, r0, u, bar_qk);
             tma_load_3d(t_kf, &tm_k, 0, r0, u, bar_qk);
             const uint8_t* sl = args.ws_slots + (size_t)t * 2 * args.slot_bytes;
             mbar_expect_tx(bar_s, 2 * 4096);
@@ -248,11 +262,11 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         const int ch = 2 * hf + c8;   // 16-byte chunk of the row: key dims 8 ch .. 8 ch + 7
                         if (ch >= DK / 8) break;
                         const uint32_t off = sw_off<64>(row, ch);
-                        const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + Y::tile + off);
+                        const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + Y::k + off);
                         const uint32_t kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
                         uint32_t kf[4], kb[4];
                         if (MODE == kLMain) {
-                            const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
+                            const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + Y::q + off);
                             const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w};
                             uint32_t qf[4], qb[4];
 #pragma unroll
@@ -266,8 +280,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                 qb[mm] = mul_bf16x2(qv[mm], pack_bf16(ey0, ey1));                                              // q~< = q e^{e}
                                 kb[mm] = mul_bf16x2(kv[mm], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
                             }
-                            *reinterpret_cast<uint4*>(bp + 2 * Y::tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
-                            *reinterpret_cast<uint4*>(bp + 3 * Y::tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
+                            *reinterpret_cast<uint4*>(bp + Y::f + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+                            *reinterpret_cast<uint4*>(bp + Y::b + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
                         } else {
 #pragma unroll
                             for (int mm = 0; mm < 4; ++mm) {
@@ -276,22 +290,11 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                 kb[mm] = mul_bf16x2(kv[mm], pack_bf16(ex2(-as_f(pb[d0]) * kLog2e), ex2(-as_f(pb[d0 + 1]) * kLog2e)));
                             }
                         }
-                        *reinterpret_cast<uint4*>(bp + 1 * Y::tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
-                        *reinterpret_cast<uint4*>(bp + 0 * Y::tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
+                        *reinterpret_cast<uint4*>(bp + Y::k + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
+                        *reinterpret_cast<uint4*>(bp + Y::kb + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
                     }
                 }
             }
-            if (MODE == kLSummary) {
-                // the q tile is not loaded in this mode: rows without tokens and padding key dims of k~< must read as zero
-                if (!row_live || DK < 32) {
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch)
-                        if (!row_live || ch >= DK / 8) *reinterpret_cast<uint4*>(bp + sw_off<64>(row, ch)) = make_uint4(0, 0, 0, 0);
-                }
-            }
-        } else if (MODE == kLSummary) {
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) *reinterpret_cast<uint4*>(bp + sw_off<64>(row, ch)) = make_uint4(0, 0, 0, 0);
         }
         fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
         handover();
@@ -309,11 +312,11 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
 
         if constexpr (MODE == kLSummary) {
-            // ---- U = [k~< | k~>]^T v -> TMEM columns [64,128); rows 0..31: backward, rows 32..63: forward ----------
+            // ---- U = [k~> | k~<]^T v -> TMEM columns [64,128); rows 0..31: forward, rows 32..63: backward ----------
             if (ctl) {
                 wait_bar(bar_v, par);
                 constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
-                const uint32_t ak = desc_lo(t_kb, Y::tile), bv = desc_lo(t_v, 16);
+                const uint32_t ak = desc_lo(t_kf, Y::tile), bv = desc_lo(t_v, 16);   // M blocks: k~>, k~< (then two tiles of no interest)
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
                     if (kk < ks) umma_ss(tmem + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
@@ -321,8 +324,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             wait_mma();
             if (wq < 2) {
-                // lane = key dim; warp 0: backward summary, warp 1: forward summary
-                const int dir = wq == 1 ? 0 : 1;
+                // lane = key dim; warp 0: forward summary, warp 1: backward summary
+                const int dir = wq;
                 const float d = ex2(totals[(dir == 0 ? 0 : 32) + lane] * kLog2e);   // decay of the whole chunk for this key dim
                 float* dst = reinterpret_cast<float*>(args.ws_slots + ((size_t)task * 2 + dir) * args.slot_bytes) + (size_t)lane * DV;
 #pragma unroll
@@ -567,9 +570,9 @@ cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     a.slot_bytes = (uint32_t)wl.slot_bytes;
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
-    size_t smem = LLayout::total + 1024;   // slack for the manual 1 KB alignment
-    const size_t rec = (size_t)rec_plan(kLThreads, DK, DV).smem_floats * 4 + 1024;
-    if (smem < rec) smem = rec;
+    const size_t rec = (size_t)rec_plan(kLThreads, DK, DV).smem_floats * 4;   // scratch of the exact recurrence (main launch only)
+    const size_t smem_sum = LLayout<kLSummary>::total;
+    const size_t smem_main = LLayout<kLMain>::total > rec ? LLayout<kLMain>::total : rec;
     // once per device: shared-memory opt-in of the two kernels and the SM count
     static std::atomic<int> sms_of[kMaxDevices];
     int dev = 0;
@@ -577,19 +580,20 @@ cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     int sms = sms_of[dev].load(std::memory_order_acquire);
     if (sms == 0) {
         cudaError_t e;
-        if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLSummary>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLMain>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLSummary>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_sum)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(bigla_long_kernel<DK, DV, kLMain>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_main)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms_of[dev].store(sms, std::memory_order_release);
     }
-    const long long cap = (long long)kLBlocksPerSm * sms;
-    const unsigned grid = (unsigned)(a.tasks < cap ? a.tasks : cap);   // persistent blocks: block b takes tasks b, b + grid, ...
-    cudaError_t le = launch_pdl(bigla_long_kernel<DK, DV, kLSummary>, dim3(grid), dim3(kLThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    // persistent blocks: block b takes tasks b, b + grid, ...
+    const long long cap_sum = (long long)kLSummaryBlocksPerSm * sms, cap_main = (long long)kLBlocksPerSm * sms;
+    const unsigned grid_sum = (unsigned)(a.tasks < cap_sum ? a.tasks : cap_sum), grid_main = (unsigned)(a.tasks < cap_main ? a.tasks : cap_main);
+    cudaError_t le = launch_pdl(bigla_long_kernel<DK, DV, kLSummary>, dim3(grid_sum), dim3(kLThreads), smem_sum, stream, tq, tk, tf, tb, tv, to, a);
     if (le == cudaSuccess)
         le = launch_pdl(bigla_long_fold_kernel<DV>, dim3((unsigned)units, 2), dim3(32 * (DV / 8)), 0, stream, a.ws_slots,
                         (const float*)a.ws_decay, a.ws_flags, (const int*)a.ws_cflags, nch, a.slot_bytes);
     if (le == cudaSuccess)
-        le = launch_pdl(bigla_long_kernel<DK, DV, kLMain>, dim3(grid), dim3(kLThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+        le = launch_pdl(bigla_long_kernel<DK, DV, kLMain>, dim3(grid_main), dim3(kLThreads), smem_main, stream, tq, tk, tf, tb, tv, to, a);
     if (le != cudaSuccess) return le;
     count_launch(3);
     return cudaGetLastError();

@@ -11,6 +11,7 @@ namespace vig {
 
 // Device status word: bit flags set by kernels whose bounded waits expire.
 constexpr int kDevStatusTimeout = 1;
+constexpr int kDevStatusInternal = 2;   // a kernel found its own set-up inconsistent (reported as VIG_ERR_CUDA)
 int* device_status_ptr();            // device address of the status word of the current device (NULL on error)
 void count_launch(unsigned n = 1);   // bumps the process-wide launch counter
 
