@@ -111,16 +111,20 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     float* dec = reinterpret_cast<float*>(bp + lay.dec);
     uint32_t mma_phase = 0;
 
-    const uint32_t t_kb = base, t_kf = base + lay.tile, t_qf = base + 2 * lay.tile, t_qb = base + 3 * lay.tile;
     const uint32_t t_v = base + lay.v;
     const uint32_t g_bytes = (uint32_t)args.rows * 128, v_bytes = (uint32_t)args.rows * 128;
-    auto load_gates_qk = [&](int unit) {
+    // The four q-type tiles form two pairs that swap roles from one unit to the next: the pair that held (q, k) - its
+    // last reader is the chunk-summary MMA - receives the next unit's log gates while this unit is still being
+    // finished, and the pair that held the log gates (then q~>, q~<) receives the next (q, k).
+    auto load_gates = [&](int unit, uint32_t pair) {
         mbar_expect_tx(bar_g, g_bytes);
-        tma_load_3d(t_qf, &tm_f, 0, 0, unit, bar_g);
-        tma_load_3d(t_qb, &tm_b, 0, 0, unit, bar_g);
+        tma_load_3d(base + pair, &tm_f, 0, 0, unit, bar_g);
+        tma_load_3d(base + pair + lay.tile, &tm_b, 0, 0, unit, bar_g);
+    };
+    auto load_qk = [&](int unit, uint32_t pair) {
         mbar_expect_tx(bar_qk, g_bytes);
-        tma_load_3d(t_kb, &tm_q, 0, 0, unit, bar_qk);
-        tma_load_3d(t_kf, &tm_k, 0, 0, unit, bar_qk);
+        tma_load_3d(base + pair, &tm_q, 0, 0, unit, bar_qk);
+        tma_load_3d(base + pair + lay.tile, &tm_k, 0, 0, unit, bar_qk);
     };
     auto load_v = [&](int unit) {
         mbar_expect_tx(bar_v, v_bytes);
@@ -146,7 +150,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid < 128) dec[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     if (tid == 0) {
-        load_gates_qk(blockIdx.x);
+        load_gates(blockIdx.x, 2 * lay.tile);
+        load_qk(blockIdx.x, 0);
         load_v(blockIdx.x);
     }
     fence_async_smem();
@@ -179,11 +184,15 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
     bool v_load_pending = false;      // control thread: the v tile of the current unit has not been requested yet
-    bool next_loads_issued = false;   // control thread: the operand tiles of the next unit are already on their way
+    bool next_gates_issued = false;   // control thread: the log gates of the next unit are already on their way
+    bool next_loads_issued = false;   // control thread: so are its q and k
     for (long long unit_ll = blockIdx.x; unit_ll < args.units; unit_ll += gridDim.x, ++it) {
         const int unit = (int)unit_ll;
         const uint32_t par = it & 1;
         const bool has_next = unit_ll + gridDim.x < args.units;
+        const uint32_t pair_qk = (it & 1) ? 2 * lay.tile : 0, pair_g = (it & 1) ? 0 : 2 * lay.tile;   // byte offsets of this unit's tile pairs
+        const uint32_t t_kb = base + pair_qk, t_kf = t_kb + lay.tile;   // q, k as loaded; k~<, k~> after scaling
+        const uint32_t t_qf = base + pair_g, t_qb = t_qf + lay.tile;    // log alpha>, log alpha< as loaded; q~>, q~< after scaling
         if (tid == 224 && has_next) {
             // pull the tiles of this block's next unit into L2
             const int pu = unit + (int)gridDim.x;
@@ -260,8 +269,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             const int ch = 2 * hf + c8;   // 16-byte chunk of the row: key dims 8 ch .. 8 ch + 7
                             if (ch >= DK / 8) break;
                             const uint32_t off = sw_off<64>(row, ch);
-                            const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + off);
-                            const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + lay.tile + off);
+                            const uint4 qv4 = *reinterpret_cast<const uint4*>(bp + pair_qk + off);
+                            const uint4 kv4 = *reinterpret_cast<const uint4*>(bp + pair_qk + lay.tile + off);
                             const uint32_t qv[4] = {qv4.x, qv4.y, qv4.z, qv4.w}, kv[4] = {kv4.x, kv4.y, kv4.z, kv4.w};
                             uint32_t qf[4], kf[4], qb[4], kb[4];
 #pragma unroll
@@ -275,10 +284,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                 qb[m] = mul_bf16x2(qv[m], pack_bf16(ey0, ey1));                                              // q~< = q e^{e}
                                 kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
                             }
-                            *reinterpret_cast<uint4*>(bp + 2 * lay.tile + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
-                            *reinterpret_cast<uint4*>(bp + 1 * lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
-                            *reinterpret_cast<uint4*>(bp + 3 * lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
-                            *reinterpret_cast<uint4*>(bp + 0 * lay.tile + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
+                            *reinterpret_cast<uint4*>(bp + pair_g + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
+                            *reinterpret_cast<uint4*>(bp + pair_qk + lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
+                            *reinterpret_cast<uint4*>(bp + pair_g + lay.tile + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
+                            *reinterpret_cast<uint4*>(bp + pair_qk + off) = make_uint4(kb[0], kb[1], kb[2], kb[3]);
                         }
                     }
                 }
@@ -378,6 +387,15 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     umma_commit(bar_mma);
                 }
                 wait_mma();
+                if (ctl && has_next) {
+                    // The summaries were the last readers of the k~ pair (chunk 1's batch included): the next unit's
+                    // log gates go there now, a good two microseconds before they are needed.
+                    wait_bar(bar_mma + 8, (it * (uint32_t)(npass_c1 + 2) + (uint32_t)npass_c1) & 1);
+                    if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
+                        load_gates(unit + (int)gridDim.x, pair_qk);
+                        next_gates_issued = true;
+                    }
+                }
                 if (warp == 1 || warp == 4) {
                     // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
                     // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
@@ -431,12 +449,14 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             wait_mma();
             if (ctl && has_next) {
-                // Every MMA that reads the four operand tiles is done once chunk 1's last batch is: the tiles of
-                // the next unit can start to load under the epilogue and the store (unless this unit must be
-                // redone by the recurrence, whose scratch overlays them).
+                // Every MMA that reads the q~ pair is done once chunk 1's last batch is: the next unit's q and k start
+                // to load under the epilogue and the store (unless this unit must be redone by the recurrence,
+                // whose scratch overlays the tiles).
                 if (nc == 2) wait_bar(bar_mma + 8, ((it + 1) * (uint32_t)(npass_c1 + 2) - 1) & 1);
                 if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
-                    load_gates_qk(unit + (int)gridDim.x);
+                    if (!next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
+                    load_qk(unit + (int)gridDim.x, pair_g);
+                    next_gates_issued = true;
                     next_loads_issued = true;
                 }
             }
@@ -485,8 +505,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (ctl) {
                 tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                if (has_next && !next_loads_issued) load_gates_qk(unit + (int)gridDim.x);
-                next_loads_issued = false;
+                if (has_next && !next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
+                if (has_next && !next_loads_issued) load_qk(unit + (int)gridDim.x, pair_g);
+                next_gates_issued = next_loads_issued = false;
                 v_load_pending = has_next;   // the v tile only once the store has read it: see above
             }
         } else {
@@ -498,7 +519,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             fence_async_smem();
             __syncthreads();
             if (ctl && has_next) {
-                load_gates_qk(unit + (int)gridDim.x);
+                load_gates(unit + (int)gridDim.x, pair_qk);
+                load_qk(unit + (int)gridDim.x, pair_g);
                 load_v(unit + (int)gridDim.x);
             }
         }
