@@ -104,6 +104,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_pfx = bar_g + 40, slot = bar_g + 48;
     volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 48);
     volatile int* time_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 52);
+    volatile int* early_gates = reinterpret_cast<volatile int*>(bp + lay.misc + 72);   // (unit counter + 1) whose next log gates went out early
     volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 56);   // [4]: range check per chunk (two used)
     const int ks_c1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;                          // K steps of chunk 1
     const int npass_c1 = ks_c1 > 4 ? 2 : 1;
@@ -135,8 +136,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0) {
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
-        mbar_init(bar_pfx, (uint32_t)nc);   // one commit per chunk issuer
+        mbar_init(bar_pfx, 2);   // one commit per direction of the prefix sums
         *time_flag = 0;
+        *early_gates = -1;
 #pragma unroll
         for (int i = 0; i < 4; ++i) slow_slot[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -180,6 +182,29 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_after();
     };
     const uint32_t row0_64 = (uint32_t)c * (kChunk * 64) >> 4, row0_128 = (uint32_t)c * (kChunk * 128) >> 4;   // in descriptor units
+    // Prefix / suffix sums of the log gates of both chunks at once (B stacks the two chunks' rows along N), issued by the
+    // chunk issuers: chunk 0's takes the forward sums, chunk 1's the backward sums (a single chunk: both).  Forward
+    // sums land in columns [0,32) (chunk 0) and [32,64) (chunk 1) of TMEM block 0, backward sums in the same columns of
+    // block 1 (a single chunk: columns [64,96) of block 0) - the columns the packed scores of the previous unit leave free.
+    const uint32_t pfx_b_col = nc == 2 ? 128u : 64u;
+    auto issue_prefix = [&](uint32_t gates_pair, bool fwd, bool bwd) {   // one commit per direction: the barrier counts two
+#pragma unroll
+        for (int dir = 0; dir < 2; ++dir) {
+            if (dir == 0 ? !fwd : !bwd) continue;
+            const uint32_t z = desc_lo(base + (dir == 0 ? lay.zf : lay.zb), 128);
+            const uint32_t g = desc_lo(base + gates_pair + (dir == 0 ? 0u : lay.tile), kChunk * 64);   // second N block = chunk 1's rows
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < ks_c0) {
+                    const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+                    const uint32_t ids = instr_desc(128, j < ks_c1 ? 64 : 32, 0, 1);   // beyond chunk 1's rows: chunk 0 alone
+                    umma_ss(tmem + (dir == 0 ? 0u : pfx_b_col), desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
+                }
+            }
+            umma_commit(bar_pfx);
+        }
+    };
+    const int npass_c0 = ks_c0 > 4 ? 2 : 1;
 
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
@@ -204,26 +229,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
 
         if (chunk_on) {
-            // ---- prefix / suffix sums of the log gates, both chunks at once: B stacks the two chunks' rows along N ----
-            // columns of TMEM block 0:  [0,32) b of chunk 0,  [32,64) b of chunk 1,  [64,96) e of chunk 0,  [96,128) e of chunk 1
-            if (issuer) {
+            // ---- prefix / suffix sums of the log gates (unless they were issued while the previous unit was finishing) ----
+            if (issuer && !(nc == 2 && *early_gates == (int)it)) {
                 wait_bar(bar_g, par);
-                // chunk 0's issuer takes the forward sums, chunk 1's the backward sums (a single chunk: both)
-#pragma unroll
-                for (int dir = 0; dir < 2; ++dir) {
-                    if (nc == 2 && dir != c) continue;
-                    const uint32_t z = desc_lo(base + (dir == 0 ? lay.zf : lay.zb), 128);
-                    const uint32_t g = desc_lo(dir == 0 ? t_qf : t_qb, kChunk * 64);   // second N block = chunk 1's rows
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (j < ks_c0) {
-                            const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                            const uint32_t ids = instr_desc(128, j < ks_c1 ? 64 : 32, 0, 1);   // beyond chunk 1's rows: chunk 0 alone
-                            umma_ss(tmem + 64 * dir, desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
-                        }
-                    }
-                }
-                umma_commit(bar_pfx);
+                issue_prefix(pair_g, nc == 1 || c == 0, nc == 1 || c == 1);   // two chunks: forward sums by chunk 0's issuer, backward by chunk 1's
             }
             wait_bar(bar_pfx, par);
             tc_fence_after();
@@ -236,18 +245,20 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const bool check_row = row_live && (row == last_row || row == c * kChunk);
                 uint32_t pf[kHalves][16], pb[kHalves][16];
                 tmem_ld16(rl + 32 * c, pf[0]);
-                tmem_ld16(rl + 64 + 32 * c, pb[0]);
+                tmem_ld16(rl + pfx_b_col + 32 * c, pb[0]);
                 tc_wait_ld();
                 if (kHalves == 2) {   // the second half travels while the first is worked on
                     tmem_ld16(rl + 32 * c + 16, pf[kHalves - 1]);
-                    tmem_ld16(rl + 64 + 32 * c + 16, pb[kHalves - 1]);
+                    tmem_ld16(rl + pfx_b_col + 32 * c + 16, pb[kHalves - 1]);
                 }
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
                     if (hf == 1) tc_wait_ld();
-                    if (hf == kHalves - 1 && c == 1) {   // chunk 0 may overwrite its TMEM block (where these sums live) from here on
+                    if (hf == kHalves - 1 && nc == 2) {
+                        // the other chunk may overwrite its TMEM block (where half of these sums live) from here on
                         tc_fence_before();
-                        asm volatile("bar.arrive 3, 256;" ::: "memory");
+                        if (c == 1) asm volatile("bar.arrive 3, 256;" ::: "memory");
+                        else asm volatile("bar.arrive 5, 256;" ::: "memory");
                     }
                     if (check_row) {
                         // totals of the log gates over the chunk: b at its last row, e at its first row.  They feed the
@@ -296,10 +307,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 asm volatile("bar.arrive 3, 256;" ::: "memory");
             }
             fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
-            if (c == 0 && nc == 2) {
-                // chunk 0's own hand-over, extended by the arrival of chunk 1's warps (they have read their sums)
+            if (nc == 2) {
+                // the chunk's own hand-over, extended by the arrival of the other chunk's warps (they have read their sums)
                 tc_fence_before();
-                named_bar(3, 2 * kChunk);
+                named_bar(c == 0 ? 3 : 5, 2 * kChunk);
                 tc_fence_after();
             } else {
                 chunk_handover();
@@ -394,6 +405,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
                         load_gates(unit + (int)gridDim.x, pair_qk);
                         next_gates_issued = true;
+                        *early_gates = (int)it + 1;   // seen by both issuers after the exchange barrier
                     }
                 }
                 if (warp == 1 || warp == 4) {
@@ -448,6 +460,15 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
+            if (tid == 224 && nc == 2 && *early_gates == (int)it + 1) {
+                // The packed scores of both chunks have been consumed (this thread has waited for chunk 1's output batch,
+                // now for chunk 0's): their TMEM columns take the next unit's prefix sums, whose log gates have been on
+                // their way since the chunk summaries.  Warp 7 has the fewest rows to write out.
+                wait_bar(bar_g + 24, ((it + 1) * (uint32_t)(npass_c0 + 2) - 1) & 1);
+                wait_bar(bar_g, par ^ 1);
+                tc_fence_after();
+                issue_prefix(pair_qk, true, true);
+            }
             if (ctl && has_next) {
                 // Every MMA that reads the q~ pair is done once chunk 1's last batch is: the next unit's q and k start
                 // to load under the epilogue and the store (unless this unit must be redone by the recurrence,
