@@ -323,6 +323,10 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
+            if (ctl && has_next && *time_flag == 0) {   // the summary batch was the last reader of every tile
+                load_operands(next);
+                load_v(next);
+            }
             if (wq < 2) {
                 // lane = key dim; warp 0: forward summary, warp 1: backward summary
                 const int dir = wq;
@@ -346,10 +350,6 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             handover();
             if (tid == 0) args.ws_cflags[task] = slow_slot[0];
             if (*time_flag != 0) break;
-            if (ctl && has_next) {
-                load_operands(next);
-                load_v(next);
-            }
         } else {
         // ---- main mode ---------------------------------------------------------------------------------------------
         // P, key columns [64 p, 64 p + 64): forward scores -> columns [0,64), backward -> [64,128)
