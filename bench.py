@@ -39,7 +39,8 @@ DEFAULT_WORKLOAD = "vig_b_224"
 # captures summarised under profiles/ (None where no capture exists yet).
 NCU_TRAFFIC_BYTES = {
     "vig_b_224": 60_383_232,    # bigla_umma_kernel<32,64>: 58.29 MB read + 2.09 MB written (profiles/bigla_umma_kernel_vig_b_224.md)
-    "vig_t_1024": 46_639_104,   # bigla_long_kernel<24,48,main>: 46.22 MB read + 0.42 MB written (profiles/bigla_long_kernels_vig_t_1024.md)
+    # vig_t_1024 runs three launches per call; their captures (profiles/bigla_long_kernels_vig_t_1024.md) were taken with
+    # flushed caches, which does not describe the L2-resident hand-over between them: no per-call figure is given.
 }
 
 

@@ -60,12 +60,15 @@ typedef enum vig_dtype { VIG_DTYPE_F32 = 0, VIG_DTYPE_BF16 = 1 } vig_dtype;
  *
  * bf16: dk in {16, 24, 32} with dv in {32, 48, 64} run on the tensor-core kernels; any other
  *       dk <= 128, dv <= 256 runs on the fp32 SIMT recurrence kernel (slow, same result
- *       contract).  Tensor-core operands are bf16 with fp32 accumulation; the running states
- *       stay on chip in fp32.  A unit whose gates decay by more than e^-60 inside one 16-token
- *       block is computed by the exact in-kernel recurrence instead of the factorised tiles.
+ *       contract).  Tensor-core operands are bf16 with fp32 accumulation; states that cross
+ *       a 128-token chunk are rounded to bf16 as tensor-core operands.  A unit whose gates decay
+ *       by more than e^-60 inside one chunk of 128 tokens is computed by the exact in-kernel
+ *       recurrence instead of the factorised tiles.
  * f32:  dk <= 128, dv <= 256; fp32 SIMT recurrence, meant for validation-sized inputs.
- * Long sequences are split into segments whose boundary states go through scratch memory that
- * the library allocates and frees on `stream` (cudaMallocAsync); use the *_ws form to supply it.
+ * Sequences of more than 256 tokens are split into 128-token chunks whose boundary states go through
+ * scratch memory that the library allocates and frees on `stream` (cudaMallocAsync); use the *_ws
+ * form to supply it.  The kernels are launched with programmatic stream serialization: each waits
+ * for the work before it in `stream` before it touches global memory.
  * Errors: NULL_POINTER, BAD_DIM, UNSUPPORTED, MISALIGNED, CUDA. */
 int vig_bigla_fwd_bf16(const void* q, const void* k, const void* v,
                        const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
@@ -116,7 +119,8 @@ int vig_bigla_fwd_static_bf16(const void* q, const void* k, const void* v,
 
 /* ---- Gate preparation (Eq. 5 line 1 / Eq. 6 lines 1-2 after the projection) ---------------------
  * log_alpha_x = logsigmoid(g_x) / tau for both directions, element-wise, evaluated in fp32 as
- * (min(g,0) - log1p(exp(-|g|))) / tau and rounded to the element type.  g_*, log_alpha_*:
+ * (min(g,0) - log1p(exp(-|g|))) / tau and rounded to the element type (the bf16 entry point takes exp
+ * and log from the special-function unit: relative error below 2e-5 before the rounding).  g_*, log_alpha_*:
  * [B,H,L,dk]; any dk >= 1; tau > 0.  In-place (log_alpha_x == g_x) is allowed.
  * Errors: NULL_POINTER, BAD_DIM, MISALIGNED, CUDA. */
 int vig_gate_prep_bf16(const void* g_fwd, const void* g_bwd,
@@ -141,14 +145,17 @@ int vig_bigla_fwd_host(const void* q, const void* k, const void* v,
 /* Static, NUL-terminated description of a vig_status value. */
 const char* vig_status_string(int status);
 /* Synchronises `stream`, then reads and clears the device status word of the current device.
- * Returns VIG_OK, VIG_ERR_DEVICE_TIMEOUT if a kernel's bounded wait on an asynchronous copy
- * expired (that unit's output is then undefined), or VIG_ERR_CUDA. */
+ * Returns VIG_OK, VIG_ERR_DEVICE_TIMEOUT if a kernel's bounded wait on an asynchronous copy or on a
+ * tensor-core batch expired (the output of that call is then undefined), or VIG_ERR_CUDA. */
 int vig_last_device_status(void* stream);
 /* Which kernel family the bf16 forward entry points use, process-wide (a testing and profiling aid:
  * all families compute the same function and meet the same tolerance).
- *   VIG_KERNEL_AUTO      tcgen05/TMEM kernel where it applies (dk in {24,32}, dv in {48,64}, L <= 256),
- *                        else the mma.sync tensor-core kernel, else the SIMT recurrence   (default)
- *   VIG_KERNEL_MMA_SYNC  never the tcgen05 kernel
+ *   VIG_KERNEL_AUTO      tcgen05/TMEM kernels for dk in {16,24,32} with dv in {32,48,64} (one persistent
+ *                        launch for L <= 256, summary / fold / main launches beyond), else the SIMT
+ *                        recurrence                                                       (default)
+ *   VIG_KERNEL_MMA_SYNC  the mma.sync tensor-core kernels instead of the tcgen05 ones.  The scratch
+ *                        size vig_bigla_workspace_bytes reports depends on this setting: query it
+ *                        under the setting the call will run with
  *   VIG_KERNEL_SIMT      always the fp32 SIMT recurrence kernel
  * Returns VIG_OK, or VIG_ERR_UNSUPPORTED for an unknown value (the setting is then unchanged). */
 #define VIG_KERNEL_AUTO 0
