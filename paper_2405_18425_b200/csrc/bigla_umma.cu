@@ -20,6 +20,10 @@
 // packing P, scaling the chunk summaries, the output epilogue.  TMEM use is 256 columns (128 per
 // chunk: prefix sums, then P, then bf16 P + U / out), shared memory about 102 KB at L = 196, so
 // two blocks share an SM and one block's MMA round trips hide behind the other's element-wise phases.
+// Blocks are persistent: block b walks over units b, b + grid, ...; the two chunks of a unit run as
+// separate pipelines (own issuing thread, own mbarrier) that meet at the prefix batch and at the
+// exchange of the chunk summaries; the operand tiles of the next unit are requested as soon as their
+// last reader of the current unit is done, and its prefix batch is issued while this unit is stored.
 #include <cuda.h>
 
 #include <atomic>
