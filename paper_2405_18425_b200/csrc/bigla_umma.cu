@@ -137,6 +137,15 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     };
 
     pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
+    if (tid == 64) {
+        // Warm L2 with this block's first unit while the kernel before this one in the stream still runs: a prefetch
+        // consumes nothing, and L2 stays coherent with whatever that kernel is still writing.
+        tma_prefetch_3d(&tm_q, 0, 0, blockIdx.x);
+        tma_prefetch_3d(&tm_k, 0, 0, blockIdx.x);
+        tma_prefetch_3d(&tm_v, 0, 0, blockIdx.x);
+        tma_prefetch_3d(&tm_f, 0, 0, blockIdx.x);
+        tma_prefetch_3d(&tm_b, 0, 0, blockIdx.x);
+    }
     if (tid == 0) {
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
