@@ -3,22 +3,28 @@
 // One thread block owns one (batch, head) unit of up to 256 tokens, split into chunks of C = 128
 // rows; thread r of the block owns token r (TMEM lane r mod 128 of chunk r / 128) in every
 // element-wise phase.  With b_t the inclusive prefix sum of log alpha> from the start of the chunk
-// and e_t the inclusive suffix sum of log alpha< to its end, Eq. 6 becomes, per chunk,
-//     [b | e] = T> la> | T< la<                      prefix sums as products with 0/1 triangular matrices
-//     q~> = q e^{b},  k~> = k e^{-b},  q~< = q e^{e},  k~< = k e^{-e}
+// and x_t the exclusive prefix sum of log alpha< (the backward decay from t to s > t is
+// exp(x_s - x_t): the gates t .. s-1), Eq. 6 becomes, per chunk,
+//     [b | x] = T [la> | la< shifted down one row]   prefix sums as one product with a 0/1 triangular matrix
+//     q~> = q e^{b},  k~> = k e^{-b},  q~< = q e^{-x},  k~< = k e^{x}
 //     P    = tril(q~> k~>^T) + triu(q~< k~<^T)
 //     U    = [k~< | k~>]^T v                          zero-input chunk summaries, both directions in one product
-//     out  = ( P v + q~> S>_in + q~< S<_in ) / 2      S>_in = U>(left chunk) * e^{b_last}, mirrored for <
+//     out  = ( P v + q~> S>_in + q~< S<_in ) / 2      S>_in = U>(left chunk) e^{b_last(left chunk)},
+//                                                     S<_in = U<(right chunk) e^{x_last(this chunk)}
+// The log alpha< tile is loaded one row low (tile row r holds the gate of token r - 1, row 0 the
+// zero fill), so its inclusive prefix sum is x; chunk 1's sums then start with the gate of token 127,
+// which is the step from chunk 0's last token into chunk 1 that the state hand-over needs.
 // Every product is a tcgen05.mma with M = 128:
 //   - the prefix sums: A = a 128-row window of a 240-row 0/1 tile ([zeros; lower triangle; ones],
-//     shifted by 16 rows per K step), B = the log-gate tile as loaded; fp32 accumulation of bf16
-//     values times 0/1 is exact up to fp32 addition;
+//     shifted by 16 rows per K step), B = both log-gate tiles of both chunks side by side along N
+//     (128 columns, one batch of eight MMAs); fp32 accumulation of bf16 values times 0/1 is exact
+//     up to fp32 addition;
 //   - P in two column halves (fwd and bwd side by side in TMEM, so the mask and the sum of the
 //     diagonal block happen in fp32), packed to bf16 and written back to TMEM as the A operand of P v;
 //   - U with A = the four operand tiles stacked along M (MN-major), q~ S with B = the bf16 state tile.
 // The threads only do element-wise work on their own row: operand scaling in place, masking and
 // packing P, scaling the chunk summaries, the output epilogue.  TMEM use is 256 columns (128 per
-// chunk: prefix sums, then P, then bf16 P + U / out), shared memory about 102 KB at L = 196, so
+// chunk: P, then bf16 P + U / out; the prefix sums of both chunks in chunk 0's), shared memory about 108 KB at L = 196, so
 // two blocks share an SM and one block's MMA round trips hide behind the other's element-wise phases.
 // Blocks are persistent: block b walks over units b, b + grid, ...; the two chunks of a unit run as
 // separate pipelines (own issuing thread, own mbarrier) that meet at the prefix batch and at the
@@ -46,23 +52,24 @@ constexpr int kMaxDevices = 64;
 
 // ---- shared-memory plan (rows = tokens of the unit rounded up to 16) ---------------------------
 struct ULayout {
-    uint32_t tile;     // bytes of one q-type tile [rows][32] bf16 (64-byte rows, 64B swizzle); four of them from offset 0:
-                       //   as loaded: q, k, log alpha>, log alpha<;  after scaling: k~<, k~>, q~>, q~<
+    uint32_t tile;     // pitch of one q-type tile [rows][32] bf16 (64-byte rows, 64B swizzle); four of them from offset 0:
+                       //   as loaded: q, k, log alpha>, log alpha< (one row low);  after scaling: k~<, k~>, q~>, q~<.
+                       //   Two chunks: the pitch is 256 rows, so that chunk 0 and chunk 1 of both gate tiles are
+                       //   four blocks at one stride, the N blocks of the prefix-sum product.
     uint32_t v;        // v tile [rows][64] bf16 (128B swizzle), later the output tile
-    uint32_t zf, zb;   // 0/1 tiles of the prefix / suffix sums
+    uint32_t zf;       // 0/1 tile of the prefix sums
     uint32_t s_fwd;    // bf16 state entering chunk 1 from the left  [32][64] (128B swizzle)
     uint32_t s_bwd;    // bf16 state entering chunk 0 from the right
-    uint32_t dec;      // [2 chunks][2][32] fp32 totals of the log gates: b at the chunk's last row, e at its first row
+    uint32_t dec;      // [2 chunks][2][32] fp32 totals of the log gates: b and x at the chunk's last row
     uint32_t misc;     // six mbarriers, TMEM slot, flags
     uint32_t total;
 };
 __host__ __device__ inline ULayout make_layout(int rows) {
     ULayout l;
-    l.tile = (uint32_t)rows * 64;
+    l.tile = rows > kChunk ? 2u * kChunk * 64u : (uint32_t)rows * 64u;
     l.v = 4 * l.tile;
     l.zf = l.v + (uint32_t)rows * 128;
-    l.zb = l.zf + kZBytes;
-    l.s_fwd = (l.zb + kZBytes + 1023u) & ~1023u;
+    l.s_fwd = (l.zf + kZBytes + 1023u) & ~1023u;
     l.s_bwd = l.s_fwd + 32 * 128;
     l.dec = l.s_bwd + 32 * 128;
     l.misc = l.dec + 4 * 32 * 4;
@@ -124,7 +131,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     auto load_gates = [&](int unit, uint32_t pair) {
         mbar_expect_tx(bar_g, g_bytes);
         tma_load_3d(base + pair, &tm_f, 0, 0, unit, bar_g);
-        tma_load_3d(base + pair + lay.tile, &tm_b, 0, 0, unit, bar_g);
+        tma_load_3d(base + pair + lay.tile, &tm_b, 0, -1, unit, bar_g);   // one row low: row 0 takes the zero fill
     };
     auto load_qk = [&](int unit, uint32_t pair) {
         mbar_expect_tx(bar_qk, g_bytes);
@@ -149,7 +156,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0) {
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
-        mbar_init(bar_pfx, 2);   // one commit per direction of the prefix sums
+        mbar_init(bar_pfx, 1);
         *time_flag = 0;
         *early_gates = -1;
 #pragma unroll
@@ -161,7 +168,18 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(kTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
-    build_zero_one_tiles(bp + lay.zf, bp + lay.zb, tid);
+    build_zero_one_tiles(bp + lay.zf, nullptr, tid);
+    // Tile rows the loads never reach (from `rows` up to the 256-row pitch) are K rows of the prefix-sum product
+    // of chunk 1: they must be finite, and nothing but the recurrence scratch ever writes them again.
+    auto zero_tail_rows = [&]() {
+        if (nc == 2) {
+            const int tail16 = (2 * kChunk - args.rows) * 4;   // 16-byte pieces per tile
+            for (int x = tid; x < 4 * tail16; x += kThreads)
+                *reinterpret_cast<uint4*>(bp + (uint32_t)(x / tail16) * lay.tile + (uint32_t)args.rows * 64 + (uint32_t)(x % tail16) * 16) =
+                    make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    zero_tail_rows();
     if (tid < 128) dec[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     if (tid == 0) {
@@ -195,27 +213,23 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_after();
     };
     const uint32_t row0_64 = (uint32_t)c * (kChunk * 64) >> 4, row0_128 = (uint32_t)c * (kChunk * 128) >> 4;   // in descriptor units
-    // Prefix / suffix sums of the log gates of both chunks at once (B stacks the two chunks' rows along N), issued by the
-    // chunk issuers: chunk 0's takes the forward sums, chunk 1's the backward sums (a single chunk: both).  Forward
-    // sums land in columns [0,32) (chunk 0) and [32,64) (chunk 1) of TMEM block 0, backward sums in the same columns of
-    // block 1 (a single chunk: columns [64,96) of block 0) - the columns the packed scores of the previous unit leave free.
-    const uint32_t pfx_b_col = nc == 2 ? 128u : 64u;
-    auto issue_prefix = [&](uint32_t gates_pair, bool fwd, bool bwd) {   // one commit per direction: the barrier counts two
+    // Prefix sums of both log-gate tiles of both chunks in one batch: B stacks, along N, the 32 key dims of
+    // [la> chunk 0 | la> chunk 1 | la< chunk 0 | la< chunk 1] (one unit of 64 or more tokens: [la> | la<]), so the
+    // sums land in TMEM block 0, columns 32 x that order - the columns the previous unit's packed scores and chunk 0's
+    // output leave free.
+    const uint32_t pfx_b_col = nc == 2 ? 64u : 32u;
+    auto issue_prefix = [&](uint32_t gates_pair) {
+        const uint32_t z = desc_lo(base + lay.zf, 128);
+        const uint32_t g = desc_lo(base + gates_pair, nc == 2 ? kChunk * 64 : lay.tile);
+        const uint32_t ids = instr_desc(128, nc == 2 ? 128 : 64, 0, 1);
 #pragma unroll
-        for (int dir = 0; dir < 2; ++dir) {
-            if (dir == 0 ? !fwd : !bwd) continue;
-            const uint32_t z = desc_lo(base + (dir == 0 ? lay.zf : lay.zb), 128);
-            const uint32_t g = desc_lo(base + gates_pair + (dir == 0 ? 0u : lay.tile), kChunk * 64);   // second N block = chunk 1's rows
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (j < ks_c0) {
-                    const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                    const uint32_t ids = instr_desc(128, j < ks_c1 ? 64 : 32, 0, 1);   // beyond chunk 1's rows: chunk 0 alone
-                    umma_ss(tmem + (dir == 0 ? 0u : pfx_b_col), desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
-                }
+        for (int j = 0; j < 8; ++j) {
+            if (j < ks_c0) {
+                const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+                umma_ss(tmem, desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
             }
-            umma_commit(bar_pfx);
         }
+        umma_commit(bar_pfx);
     };
     const int npass_c0 = ks_c0 > 4 ? 2 : 1;
 
@@ -243,9 +257,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
         if (chunk_on) {
             // ---- prefix / suffix sums of the log gates (unless they were issued while the previous unit was finishing) ----
-            if (issuer && !(nc == 2 && *early_gates == (int)it)) {
+            if (issuer && c == 0 && !(nc == 2 && *early_gates == (int)it)) {
                 wait_bar(bar_g, par);
-                issue_prefix(pair_g, nc == 1 || c == 0, nc == 1 || c == 1);   // two chunks: forward sums by chunk 0's issuer, backward by chunk 1's
+                issue_prefix(pair_g);
             }
             wait_bar(bar_pfx, par);
             tc_fence_after();
@@ -255,7 +269,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (warp_live) {
                 constexpr int kHalves = (DK + 15) / 16;
                 const int last_row = min(L, (c + 1) * kChunk) - 1;
-                const bool check_row = row_live && (row == last_row || row == c * kChunk);
+                const bool check_row = row == last_row;
                 uint32_t pf[kHalves][16], pb[kHalves][16];
                 tmem_ld16(rl + 32 * c, pf[0]);
                 tmem_ld16(rl + pfx_b_col + 32 * c, pb[0]);
@@ -267,24 +281,18 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
                     if (hf == 1) tc_wait_ld();
-                    if (hf == kHalves - 1 && nc == 2) {
-                        // the other chunk may overwrite its TMEM block (where half of these sums live) from here on
+                    if (hf == kHalves - 1 && nc == 2 && c == 1) {
+                        // chunk 0 may overwrite its TMEM block (where these sums live) from here on
                         tc_fence_before();
-                        if (c == 1) asm volatile("bar.arrive 3, 256;" ::: "memory");
-                        else asm volatile("bar.arrive 5, 256;" ::: "memory");
+                        asm volatile("bar.arrive 3, 256;" ::: "memory");
                     }
                     if (check_row) {
-                        // totals of the log gates over the chunk: b at its last row, e at its first row.  They feed the
-                        // range check (done by a whole warp after the hand-over) and the decay of the chunk summaries.
-                        if (row == last_row) {
+                        // totals of the log gates over the chunk, b and x at its last row.  They feed the range check
+                        // (done by a whole warp after the hand-over) and the decay of the chunk summaries.
 #pragma unroll
-                            for (int x = 0; x < 4; ++x)
-                                reinterpret_cast<uint4*>(dec + (2 * c) * 32 + 16 * hf)[x] = make_uint4(pf[hf][4 * x], pf[hf][4 * x + 1], pf[hf][4 * x + 2], pf[hf][4 * x + 3]);
-                        }
-                        if (row == c * kChunk) {
-#pragma unroll
-                            for (int x = 0; x < 4; ++x)
-                                reinterpret_cast<uint4*>(dec + (2 * c + 1) * 32 + 16 * hf)[x] = make_uint4(pb[hf][4 * x], pb[hf][4 * x + 1], pb[hf][4 * x + 2], pb[hf][4 * x + 3]);
+                        for (int x = 0; x < 4; ++x) {
+                            reinterpret_cast<uint4*>(dec + (2 * c) * 32 + 16 * hf)[x] = make_uint4(pf[hf][4 * x], pf[hf][4 * x + 1], pf[hf][4 * x + 2], pf[hf][4 * x + 3]);
+                            reinterpret_cast<uint4*>(dec + (2 * c + 1) * 32 + 16 * hf)[x] = make_uint4(pb[hf][4 * x], pb[hf][4 * x + 1], pb[hf][4 * x + 2], pb[hf][4 * x + 3]);
                         }
                     }
                     if (row_live) {
@@ -305,8 +313,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                 const float ey0 = ex2(as_f(pb[hf][d0]) * kLog2e), ey1 = ex2(as_f(pb[hf][d0 + 1]) * kLog2e);
                                 qf[m] = mul_bf16x2(qv[m], pack_bf16(ex0, ex1));                                              // q~> = q e^{b}
                                 kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
-                                qb[m] = mul_bf16x2(qv[m], pack_bf16(ey0, ey1));                                              // q~< = q e^{e}
-                                kb[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
+                                qb[m] = mul_bf16x2(qv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // q~< = q e^{-x}
+                                kb[m] = mul_bf16x2(kv[m], pack_bf16(ey0, ey1));                                              // k~< = k e^{x}
                             }
                             *reinterpret_cast<uint4*>(bp + pair_g + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
                             *reinterpret_cast<uint4*>(bp + pair_qk + lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
@@ -320,16 +328,17 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 asm volatile("bar.arrive 3, 256;" ::: "memory");
             }
             fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
-            if (nc == 2) {
-                // the chunk's own hand-over, extended by the arrival of the other chunk's warps (they have read their sums)
+            if (nc == 2 && c == 0) {
+                // the chunk's own hand-over, extended by the arrival of chunk 1's warps (they have read their sums)
+                asm volatile("bar.arrive 5, 160;" ::: "memory");   // chunk 0's totals are written: see the chunk summaries
                 tc_fence_before();
-                named_bar(c == 0 ? 3 : 5, 2 * kChunk);
+                named_bar(3, 2 * kChunk);
                 tc_fence_after();
             } else {
                 chunk_handover();
             }
             if (wq == 2) {
-                // range check, one key dim per lane: b is smallest at the last row of the chunk, e at its first row
+                // range check, one key dim per lane: b and x are smallest at the last row of the chunk
                 const bool out_of_range = dec[(2 * c) * 32 + lane] < -kGateRange || dec[(2 * c + 1) * 32 + lane] < -kGateRange;
                 const bool any = __any_sync(0xffffffffu, out_of_range);
                 if (lane == 0) slow_slot[c] = any ? 1 : 0;
@@ -423,8 +432,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
                 if (warp == 1 || warp == 4) {
                     // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
-                    // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state for chunk 0
-                    const float d = ex2(dec[(warp == 1 ? 0 : 96) + lane] * kLog2e);   // decay of the whole chunk for key dim `lane`
+                    // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state
+                    // for chunk 0.  Both are scaled by chunk 0's total decay of their direction, for key dim `lane`.
+                    if (warp == 4) named_bar(5, 160);   // chunk 0's threads arrived after writing their totals
+                    const float d = ex2(dec[(warp == 1 ? 0 : 32) + lane] * kLog2e);
                     uint8_t* st = bp + (warp == 1 ? lay.s_fwd : lay.s_bwd);
 #pragma unroll
                     for (int hb = 0; hb < 2; ++hb) {
@@ -479,8 +490,13 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // their way since the chunk summaries.  Warp 7 has the fewest rows to write out.
                 wait_bar(bar_g + 24, ((it + 1) * (uint32_t)(npass_c0 + 2) - 1) & 1);
                 wait_bar(bar_g, par ^ 1);
+            }
+            if (nc == 2 && warp == 7) {
+                // ... and chunk 0's output has left TMEM block 0, which takes the sums of all four gate blocks
+                named_bar(6, 160);
                 tc_fence_after();
-                issue_prefix(pair_qk, true, true);
+                if (lane == 0 && *early_gates == (int)it + 1) issue_prefix(pair_qk);
+                __syncwarp();
             }
             if (ctl && has_next) {
                 // Every MMA that reads the q~ pair is done once chunk 1's last batch is: the next unit's q and k start
@@ -496,33 +512,28 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
             if (warp_live) {
-#pragma unroll
-                for (int hb = 0; hb < DV / 32; ++hb) {
-                    uint32_t r[32];
-                    tmem_ld32(rc + 64 + hb * 32, r);
-                    tc_wait_ld();
-                    if (row_live) {
-#pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
-                            uint32_t o[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
-                            *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
-                        }
-                    }
-                }
+                uint32_t r[2][32];
+                tmem_ld32(rc + 64, r[0]);
+                if (DV == 64) tmem_ld32(rc + 96, r[1]);
                 if (DV == 48) {
-                    uint32_t r[16];
-                    tmem_ld16(rc + 64 + 32, r);
-                    tc_wait_ld();
-                    if (row_live) {
+                    uint32_t t[16];
+                    tmem_ld16(rc + 96, t);
 #pragma unroll
-                        for (int ch = 0; ch < 2; ++ch) {
-                            uint32_t o[4];
+                    for (int e = 0; e < 16; ++e) r[1][e] = t[e];
+                }
+                tc_wait_ld();
+                if (nc == 2 && c == 0) {   // TMEM block 0 is free for the next unit's prefix sums
+                    tc_fence_before();
+                    asm volatile("bar.arrive 6, 160;" ::: "memory");
+                }
+                if (row_live) {
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
-                            *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
-                        }
+                    for (int ch = 0; ch < DV / 8; ++ch) {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            o[e] = pack_bf16(0.5f * as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e]), 0.5f * as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e + 1]));
+                        *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
             }
@@ -550,6 +561,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const size_t ok = (size_t)unit * L * DK, ov = (size_t)unit * L * DV;
             recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
                                            args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));
+            __syncthreads();
+            zero_tail_rows();
             fence_async_smem();
             __syncthreads();
             if (ctl && has_next) {

@@ -143,10 +143,11 @@ __device__ __forceinline__ float fast_rcp(float x) {
 }
 constexpr int kRcpSteps = 1;
 
-// Builds the two 240-row 0/1 tiles of the prefix / suffix sums (K-major without swizzle: 8-row groups of 256
+// Builds the 240-row 0/1 tiles of the prefix / suffix sums (K-major without swizzle: 8-row groups of 256
 // bytes, each two 8x8 core matrices for K 0..7 and K 8..15).  Rows 0..111 of `zf` are zeros, rows 112..127 the
-// lower triangle (diagonal included), rows 128..239 ones; `zb` holds ones, the upper triangle, zeros.  The
-// 128-row window starting at row 112 - 16 j is the operand of K step j.  Threads 0..239 of the block write.
+// lower triangle (diagonal included), rows 128..239 ones; `zb` (may be null: not built) holds ones, the upper
+// triangle, zeros.  The 128-row window starting at row 112 - 16 j is the operand of K step j.  Threads 0..239
+// of the block write.
 __device__ __forceinline__ void build_zero_one_tiles(uint8_t* zf, uint8_t* zb, int tid) {
     if (tid < (int)kZRows) {
         uint32_t f[8], b[8];
@@ -167,8 +168,10 @@ __device__ __forceinline__ void build_zero_one_tiles(uint8_t* zf, uint8_t* zb, i
         const uint32_t off = (uint32_t)(tid >> 3) * 256 + (uint32_t)(tid & 7) * 16;
         *reinterpret_cast<uint4*>(zf + off) = make_uint4(f[0], f[1], f[2], f[3]);
         *reinterpret_cast<uint4*>(zf + off + 128) = make_uint4(f[4], f[5], f[6], f[7]);
-        *reinterpret_cast<uint4*>(zb + off) = make_uint4(b[0], b[1], b[2], b[3]);
-        *reinterpret_cast<uint4*>(zb + off + 128) = make_uint4(b[4], b[5], b[6], b[7]);
+        if (zb) {
+            *reinterpret_cast<uint4*>(zb + off) = make_uint4(b[0], b[1], b[2], b[3]);
+            *reinterpret_cast<uint4*>(zb + off + 128) = make_uint4(b[4], b[5], b[6], b[7]);
+        }
     }
 }
 
