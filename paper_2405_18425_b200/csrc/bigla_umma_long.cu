@@ -3,11 +3,13 @@
 // The sequence of every (batch, head) unit is cut into chunks of 128 tokens; a task is one chunk, and the
 // running states of Eq. 6 that cross chunk boundaries travel through scratch memory in three launches:
 //   1. summary: per chunk, the state a zero input would leave behind, U> = diag(e^{b_last}) (k~>)^T v and
-//      U< = diag(e^{e_first}) (k~<)^T v, and the chunk's decay d> = e^{b_last}, d< = e^{e_first}
-//      (b, e: prefix / suffix sums of the log gates inside the chunk, as in the single-block kernel);
-//   2. fold: S>_in(m + 1) = d>(m) S>_in(m) + U>(m) from the left, S<_in(m - 1) = d<(m) S<_in(m) + U<(m) from the
-//      right, in fp32; every incoming state is written back over its summary as the bf16 shared-memory image
-//      the next launch copies in with one bulk copy;
+//      U< = (k~<)^T v, and the chunk's decay d> = e^{b_last}, d< = e^{x_last}
+//      (b: inclusive prefix sums of log alpha> inside the chunk, x: exclusive prefix sums of log alpha< - its tile
+//      is loaded one row low, so chunk m's sums start with the gate of the token before it, the step across the
+//      chunk boundary -, k~> = k e^{-b}, k~< = k e^{x}, as in the single-block kernel);
+//   2. fold: S>_in(m + 1) = d>(m) S>_in(m) + U>(m) from the left; from the right R(m) = U<(m) + d<(m) R(m + 1) and
+//      S<_in(m) = d<(m) R(m + 1) (q~< = q e^{-x} lacks the chunk's own decay), in fp32; every incoming state is
+//      written back over its summary as the bf16 shared-memory image the next launch copies in with one bulk copy;
 //   3. main: per chunk, out = ( P v + q~> S>_in + q~< S<_in ) / 2 with P = tril(q~> k~>^T) + triu(q~< k~<^T).
 // Blocks are persistent (three per SM, 128 threads, 128 TMEM columns each) and walk over the tasks; thread r
 // owns token r of the chunk in every element-wise phase.  All products are tcgen05.mma with M = 128.
@@ -52,7 +54,7 @@ LongWs long_ws_layout(long long units, int nch, int dv) {
 
 // ---- shared memory -------------------------------------------------------------------------------------------
 // Main mode holds four q-type tiles [128][32] bf16 (64B swizzle; loaded: q, k, log alpha>, log alpha<; scaled in
-// place: k~<, k~>, q~>, q~<), the v tile (later the output tile), the 0/1 tiles and the two incoming states.
+// place: k~<, k~>, q~>, q~<), the v tile (later the output tile), the 0/1 tile and the two incoming states.
 // Summary mode needs neither q nor states and writes k~< over the log alpha> tile once the prefix sums are taken,
 // which keeps a block below a quarter of an SM's shared memory.
 template <int MODE>
@@ -65,10 +67,9 @@ struct LLayout {
     static constexpr uint32_t kb = MODE == kLMain ? q : f;                // where k~< lives
     static constexpr uint32_t v = b + tile;                               // v tile [128][64] bf16 (128B swizzle)
     static constexpr uint32_t zf = v + 128 * 128;
-    static constexpr uint32_t zb = zf + kZBytes;
-    static constexpr uint32_t s_fwd = (zb + kZBytes + 1023u) & ~1023u;    // main only: incoming states, bf16 [32][64], 128B swizzle
+    static constexpr uint32_t s_fwd = (zf + kZBytes + 1023u) & ~1023u;    // main only: incoming states, bf16 [32][64], 128B swizzle
     static constexpr uint32_t s_bwd = s_fwd + 4096;
-    static constexpr uint32_t misc = MODE == kLMain ? s_bwd + 4096 : zb + kZBytes;   // mbarriers, TMEM slot, flags, totals
+    static constexpr uint32_t misc = MODE == kLMain ? s_bwd + 4096 : zf + kZBytes;   // mbarriers, TMEM slot, flags, totals
     static constexpr uint32_t total = misc + 64 + 256;
 };
 
@@ -115,7 +116,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + Y::misc + 40);
     volatile int* time_flag = reinterpret_cast<volatile int*>(bp + Y::misc + 44);
     volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + Y::misc + 48);   // range check of the chunk (summary mode)
-    float* totals = reinterpret_cast<float*>(bp + Y::misc + 64);   // [2][32] chunk totals of the log gates: b at the last row, e at the first row
+    float* totals = reinterpret_cast<float*>(bp + Y::misc + 64);   // [2][32] chunk totals of the log gates: b and x at the last row
     uint32_t mma_phase = 0;
 
     const uint32_t t_kb = base + Y::kb, t_kf = base + Y::k, t_qf = base + Y::f, t_qb = base + Y::b, t_q = base + Y::q;
@@ -127,7 +128,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const int u = task_unit(t), r0 = task_chunk(t) * kChunk;
         mbar_expect_tx(bar_g, 2 * Y::tile);
         tma_load_3d(t_qf, &tm_f, 0, r0, u, bar_g);
-        tma_load_3d(t_qb, &tm_b, 0, r0, u, bar_g);
+        tma_load_3d(t_qb, &tm_b, 0, r0 - 1, u, bar_g);   // one row low (row -1 of the unit: the zero fill)
         if (MODE == kLMain) {
             mbar_expect_tx(bar_qk, 2 * Y::tile);
             tma_load_3d(t_q, &tm_q, 0, r0, u, bar_qk);
@@ -169,9 +170,9 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(kLTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
-    // the 240 rows of the 0/1 tiles, two passes of 128 threads
-    build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid);
-    build_zero_one_tiles(bp + Y::zf, bp + Y::zb, tid + kLThreads);
+    // the 240 rows of the 0/1 tile, two passes of 128 threads
+    build_zero_one_tiles(bp + Y::zf, nullptr, tid);
+    build_zero_one_tiles(bp + Y::zf, nullptr, tid + kLThreads);
     if (tid < 64) totals[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     fence_async_smem();
@@ -223,18 +224,17 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (MODE == kLMain) tma_prefetch_3d(&tm_q, 0, pr, pu);
         }
 
-        // ---- prefix / suffix sums of the log gates -> TMEM columns [0,32) / [32,64) -----------------------------
+        // ---- prefix sums of both log-gate tiles (side by side along N) -> TMEM columns [0,32) / [32,64) ----------
         if (ctl) {
             wait_bar(bar_g, par);
-            constexpr uint32_t kIdS = instr_desc(128, 32, 0, 1);
-            const uint32_t zf = desc_lo(base + Y::zf, 128), zb = desc_lo(base + Y::zb, 128);
-            const uint32_t gf = desc_lo(t_qf, 16), gb = desc_lo(t_qb, 16);
+            constexpr uint32_t kIdS = instr_desc(128, 64, 0, 1);
+            const uint32_t zf = desc_lo(base + Y::zf, 128);
+            const uint32_t g = desc_lo(t_qf, Y::tile);   // second N block: the log alpha< tile
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 if (j < ks) {
                     const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                    umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(gf + j * 64, kHiK64), kIdS, j > 0);
-                    umma_ss(tmem + 32, desc64(zb + win, kHiZ), desc64(gb + j * 64, kHiK64), kIdS, j > 0);
+                    umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(g + j * 64, kHiK64), kIdS, j > 0);
                 }
             }
             umma_commit(bar_mma);
@@ -245,7 +245,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // ---- scaled operands, in place: every thread rewrites its own row -----------------------------------------
         if (warp_live) {
             constexpr int kHalves = (DK + 15) / 16;
-            const bool check_row = row_live && (row == rows_here - 1 || row == 0);
+            const bool check_row = row == rows_here - 1;
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) {
                 uint32_t pf[16], pb[16];
@@ -253,17 +253,12 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tmem_ld16(rc + 32 + 16 * hf, pb);
                 tc_wait_ld();
                 if (check_row) {
-                    // totals of the log gates over the chunk: b at its last row, e at its first row (range check after
-                    // the hand-over, decay of the summary)
-                    if (row == rows_here - 1) {
+                    // totals of the log gates over the chunk, b and x at its last row (range check after the hand-over,
+                    // decay of the summary)
 #pragma unroll
-                        for (int x = 0; x < 4; ++x)
-                            reinterpret_cast<uint4*>(totals + 16 * hf)[x] = make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
-                    }
-                    if (row == 0) {
-#pragma unroll
-                        for (int x = 0; x < 4; ++x)
-                            reinterpret_cast<uint4*>(totals + 32 + 16 * hf)[x] = make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3]);
+                    for (int x = 0; x < 4; ++x) {
+                        reinterpret_cast<uint4*>(totals + 16 * hf)[x] = make_uint4(pf[4 * x], pf[4 * x + 1], pf[4 * x + 2], pf[4 * x + 3]);
+                        reinterpret_cast<uint4*>(totals + 32 + 16 * hf)[x] = make_uint4(pb[4 * x], pb[4 * x + 1], pb[4 * x + 2], pb[4 * x + 3]);
                     }
                 }
                 if (row_live) {
@@ -287,8 +282,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                 const float ey0 = ex2(as_f(pb[d0]) * kLog2e), ey1 = ex2(as_f(pb[d0 + 1]) * kLog2e);
                                 qf[mm] = mul_bf16x2(qv[mm], pack_bf16(ex0, ex1));                                              // q~> = q e^{b}
                                 kf[mm] = mul_bf16x2(kv[mm], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
-                                qb[mm] = mul_bf16x2(qv[mm], pack_bf16(ey0, ey1));                                              // q~< = q e^{e}
-                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // k~< = k e^{-e}
+                                qb[mm] = mul_bf16x2(qv[mm], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // q~< = q e^{-x}
+                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(ey0, ey1));                                              // k~< = k e^{x}
                             }
                             *reinterpret_cast<uint4*>(bp + Y::f + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
                             *reinterpret_cast<uint4*>(bp + Y::b + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
@@ -297,7 +292,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             for (int mm = 0; mm < 4; ++mm) {
                                 const int d0 = 8 * c8 + 2 * mm;
                                 kf[mm] = mul_bf16x2(kv[mm], pack_bf16(ex2(-as_f(pf[d0]) * kLog2e), ex2(-as_f(pf[d0 + 1]) * kLog2e)));
-                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(ex2(-as_f(pb[d0]) * kLog2e), ex2(-as_f(pb[d0 + 1]) * kLog2e)));
+                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(ex2(as_f(pb[d0]) * kLog2e), ex2(as_f(pb[d0 + 1]) * kLog2e)));
                             }
                         }
                         *reinterpret_cast<uint4*>(bp + Y::k + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);
@@ -309,7 +304,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
         handover();
         if (wq == 2 && MODE == kLSummary) {
-            // range check, one key dim per lane: b is smallest at the last row of the chunk, e at its first row
+            // range check, one key dim per lane: b and x are smallest at the last row of the chunk
             const bool out_of_range = totals[lane] < -kGateRange || totals[32 + lane] < -kGateRange;
             const bool any = __any_sync(0xffffffffu, out_of_range);
             if (lane == 0) slow_slot[0] = any ? 1 : 0;
@@ -341,6 +336,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // lane = key dim; warp 0: forward summary, warp 1: backward summary
                 const int dir = wq;
                 const float d = ex2(totals[(dir == 0 ? 0 : 32) + lane] * kLog2e);   // decay of the whole chunk for this key dim
+                const float us = dir == 0 ? d : 1.f;   // the forward summary carries the chunk's decay, the backward one does not
                 float* dst = reinterpret_cast<float*>(args.ws_slots + ((size_t)task * 2 + dir) * args.slot_bytes) + (size_t)lane * DV;
 #pragma unroll
                 for (int hb = 0; hb < 2; ++hb) {
@@ -352,7 +348,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int x = 0; x < 8; ++x) {
                         if (hb * 32 + 4 * x < DV)
                             reinterpret_cast<float4*>(dst + hb * 32)[x] =
-                                make_float4(as_f(r[4 * x]) * d, as_f(r[4 * x + 1]) * d, as_f(r[4 * x + 2]) * d, as_f(r[4 * x + 3]) * d);
+                                make_float4(as_f(r[4 * x]) * us, as_f(r[4 * x + 1]) * us, as_f(r[4 * x + 2]) * us, as_f(r[4 * x + 3]) * us);
                     }
                 }
                 args.ws_decay[((size_t)task * 2 + dir) * 32 + lane] = d;
@@ -545,6 +541,11 @@ bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, int* ws_flags, 
             if (mb + b < nch) {
                 const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
                 uint8_t* img = ws_slots + (((size_t)unit * nch + m) * 2 + dir) * slot_bytes;
+                // forward: the state entering chunk m is the carry; backward: the carry times the chunk's own decay
+                if (dir == 1) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) carry[e] *= d[b];
+                }
                 uint4 o;
                 o.x = pack_bf16(carry[0], carry[1]); o.y = pack_bf16(carry[2], carry[3]);
                 o.z = pack_bf16(carry[4], carry[5]); o.w = pack_bf16(carry[6], carry[7]);
@@ -553,7 +554,7 @@ bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, int* ws_flags, 
                     *reinterpret_cast<uint4*>(img + i * 128 + (((CPR + c) ^ (i & 7)) << 4)) = make_uint4(0, 0, 0, 0);
                 const float uu[8] = {u[b][0].x, u[b][0].y, u[b][0].z, u[b][0].w, u[b][1].x, u[b][1].y, u[b][1].z, u[b][1].w};
 #pragma unroll
-                for (int e = 0; e < 8; ++e) carry[e] = fmaf(carry[e], d[b], uu[e]);
+                for (int e = 0; e < 8; ++e) carry[e] = dir == 0 ? fmaf(carry[e], d[b], uu[e]) : carry[e] + uu[e];
             }
         }
     }
