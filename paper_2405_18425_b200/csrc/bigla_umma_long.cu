@@ -29,7 +29,7 @@ using namespace umma;
 
 constexpr int kLThreads = 128;
 constexpr uint32_t kLTmemCols = 128;
-constexpr int kLBlocksPerSm = 3;          // main launch: blocks per SM (shared memory)
+constexpr int kLBlocksPerSm = 4;          // main launch: blocks per SM (shared memory, registers and TMEM: 4 x 128 columns)
 constexpr int kLSummaryBlocksPerSm = 4;   // summary launch (shared memory and TMEM: 4 x 128 columns)
 constexpr int kMaxDevices = 64;
 enum LongMode { kLMain = 0, kLSummary = 1 };
@@ -54,7 +54,8 @@ LongWs long_ws_layout(long long units, int nch, int dv) {
 
 // ---- shared memory -------------------------------------------------------------------------------------------
 // Main mode holds four q-type tiles [128][32] bf16 (64B swizzle; loaded: q, k, log alpha>, log alpha<; scaled in
-// place: k~<, k~>, q~>, q~<), the v tile (later the output tile), the 0/1 tile and the two incoming states.
+// place: k~<, k~>, q~>, q~<), the v tile (later the output tile) and the 0/1 tile; the two incoming states (4 KB
+// each) land on the first 64 rows of the k~> and k~< tiles once the first score batch, their last reader, is done.
 // Summary mode needs neither q nor states and writes k~< over the log alpha> tile once the prefix sums are taken,
 // which keeps a block below a quarter of an SM's shared memory.
 template <int MODE>
@@ -67,9 +68,9 @@ struct LLayout {
     static constexpr uint32_t kb = MODE == kLMain ? q : f;                // where k~< lives
     static constexpr uint32_t v = b + tile;                               // v tile [128][64] bf16 (128B swizzle)
     static constexpr uint32_t zf = v + 128 * 128;
-    static constexpr uint32_t s_fwd = (zf + kZBytes + 1023u) & ~1023u;    // main only: incoming states, bf16 [32][64], 128B swizzle
-    static constexpr uint32_t s_bwd = s_fwd + 4096;
-    static constexpr uint32_t misc = MODE == kLMain ? s_bwd + 4096 : zf + kZBytes;   // mbarriers, TMEM slot, flags, totals
+    static constexpr uint32_t s_fwd = k;                                  // main only: incoming states, bf16 [32][64], 128B swizzle,
+    static constexpr uint32_t s_bwd = q;                                  //   over rows 0..63 of k~> / k~< after the first score batch
+    static constexpr uint32_t misc = zf + kZBytes;                        // mbarriers, TMEM slot, flags, totals
     static constexpr uint32_t total = misc + 64 + 256;
 };
 
@@ -133,14 +134,16 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_expect_tx(bar_qk, 2 * Y::tile);
             tma_load_3d(t_q, &tm_q, 0, r0, u, bar_qk);
             tma_load_3d(t_kf, &tm_k, 0, r0, u, bar_qk);
-            const uint8_t* sl = args.ws_slots + (size_t)t * 2 * args.slot_bytes;
-            mbar_expect_tx(bar_s, 2 * 4096);
-            bulk_load_1d(base + Y::s_fwd, sl, 4096, bar_s);
-            bulk_load_1d(base + Y::s_bwd, sl + args.slot_bytes, 4096, bar_s);
         } else {
             mbar_expect_tx(bar_qk, Y::tile);
             tma_load_3d(t_kf, &tm_k, 0, r0, u, bar_qk);
         }
+    };
+    auto load_states = [&](long long t) {
+        const uint8_t* sl = args.ws_slots + (size_t)t * 2 * args.slot_bytes;
+        mbar_expect_tx(bar_s, 2 * 4096);
+        bulk_load_1d(base + Y::s_fwd, sl, 4096, bar_s);
+        bulk_load_1d(base + Y::s_bwd, sl + args.slot_bytes, 4096, bar_s);
     };
     auto load_v = [&](long long t) {
         mbar_expect_tx(bar_v, 128 * 128);
@@ -375,6 +378,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
+            if (p == 0 && ctl) load_states(task);   // rows 0..63 of k~> and k~< have been read for the last time
             if (warp_live) {
                 uint32_t pk[16];
                 combine_any(2 * p, wq, true, rc, rc + 64, lane, pk);
