@@ -218,15 +218,6 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // a unit whose gates left the factorised range (found by the summary launch) is redone by the recurrence
         const bool unit_slow = MODE == kLMain && args.ws_flags[unit] != 0;
 
-        if (tid == 96 && has_next) {   // pull the next task's tiles into L2
-            const int pu = task_unit(next), pr = task_chunk(next) * kChunk;
-            tma_prefetch_3d(&tm_f, 0, pr, pu);
-            tma_prefetch_3d(&tm_b, 0, pr, pu);
-            tma_prefetch_3d(&tm_k, 0, pr, pu);
-            tma_prefetch_3d(&tm_v, 0, pr, pu);
-            if (MODE == kLMain) tma_prefetch_3d(&tm_q, 0, pr, pu);
-        }
-
         // ---- prefix sums of both log-gate tiles (side by side along N) -> TMEM columns [0,32) / [32,64) ----------
         if (ctl) {
             wait_bar(bar_g, par);
