@@ -9,7 +9,7 @@
 //      chunk boundary -, k~> = k e^{-b}, k~< = k e^{x}, as in the single-block kernel);
 //   2. fold: S>_in(m + 1) = d>(m) S>_in(m) + U>(m) from the left; from the right R(m) = U<(m) + d<(m) R(m + 1) and
 //      S<_in(m) = d<(m) R(m + 1) (q~< = q e^{-x} lacks the chunk's own decay), in fp32; every incoming state is
-//      written back over its summary as the bf16 shared-memory image the next launch copies in with one bulk copy;
+//      written out as the bf16 shared-memory image the next launch copies in with one bulk copy;
 //   3. main: per chunk, out = ( P v + q~> S>_in + q~< S<_in ) / 2 with P = tril(q~> k~>^T) + triu(q~< k~<^T).
 // Blocks are persistent (three per SM, 128 threads, 128 TMEM columns each) and walk over the tasks; thread r
 // owns token r of the chunk in every element-wise phase.  All products are tcgen05.mma with M = 128.
@@ -35,17 +35,20 @@ constexpr int kMaxDevices = 64;
 enum LongMode { kLMain = 0, kLSummary = 1 };
 
 // ---- scratch ---------------------------------------------------------------------------------------------
-// slot(unit, chunk, dir): 32 x DV fp32 (summary, key dim major), overwritten by the fold with a 4 KB bf16 tile
-// image [32][64] (128-byte rows, 128B swizzle);  decay(unit, chunk, dir): 32 fp32;  flags(unit), chunk flags(unit, chunk): int.
+// slot(unit, chunk, dir): 32 x DV fp32 (summary, key dim major);  image(unit, chunk, dir): the incoming state as a 4 KB
+// bf16 tile [32][64] (128-byte rows, 128B swizzle), written by the fold;  decay(unit, chunk, dir): 32 fp32;
+// flags(unit), chunk flags(unit, chunk): int.
 // Every word is written before it is read within one call: nothing has to be cleared beforehand.
 struct LongWs {
-    size_t slot_bytes, decay_off, flags_off, cflags_off, total;
+    size_t slot_bytes, img_off, decay_off, flags_off, cflags_off, total;
 };
+constexpr size_t kImgBytes = 4096;
 LongWs long_ws_layout(long long units, int nch, int dv) {
     LongWs w;
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-    w.slot_bytes = (size_t)32 * dv * 4 < 4096 ? 4096 : (size_t)32 * dv * 4;
-    w.decay_off = up((size_t)units * nch * 2 * w.slot_bytes);
+    w.slot_bytes = (size_t)32 * dv * 4;
+    w.img_off = up((size_t)units * nch * 2 * w.slot_bytes);
+    w.decay_off = w.img_off + up((size_t)units * nch * 2 * kImgBytes);
     w.flags_off = w.decay_off + up((size_t)units * nch * 2 * 32 * 4);
     w.cflags_off = w.flags_off + up((size_t)units * 4);
     w.total = w.cflags_off + up((size_t)units * nch * 4);
@@ -80,6 +83,7 @@ struct LArgs {
     int L, nch;
     long long tasks;
     uint8_t* ws_slots;    // [units][nch][2][slot_bytes]
+    uint8_t* ws_img;      // [units][nch][2][4096]
     float* ws_decay;      // [units][nch][2][32]
     int* ws_flags;        // [units]: the unit needs the exact recurrence (written by the fold launch)
     int* ws_cflags;       // [units][nch]: per-chunk range check of the summary launch
@@ -140,10 +144,10 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
     };
     auto load_states = [&](long long t) {
-        const uint8_t* sl = args.ws_slots + (size_t)t * 2 * args.slot_bytes;
+        const uint8_t* im = args.ws_img + (size_t)t * 2 * kImgBytes;
         mbar_expect_tx(bar_s, 2 * 4096);
-        bulk_load_1d(base + Y::s_fwd, sl, 4096, bar_s);
-        bulk_load_1d(base + Y::s_bwd, sl + args.slot_bytes, 4096, bar_s);
+        bulk_load_1d(base + Y::s_fwd, im, 4096, bar_s);
+        bulk_load_1d(base + Y::s_bwd, im + kImgBytes, 4096, bar_s);
     };
     auto load_v = [&](long long t) {
         mbar_expect_tx(bar_v, 128 * 128);
@@ -495,61 +499,58 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0 && *time_flag != 0) atomicOr(args.dev_status, kDevStatusTimeout);
 }
 
-// Sequential fold of the chunk summaries of one unit and direction.  Thread (i, c) owns the eight value dims
-// 8 c .. 8 c + 7 of key dim i.  Chunks are taken in batches of sixteen so that their loads are all in flight
-// together; after a batch is in registers the incoming states are written, as bf16 tile images, over the
-// first 4 KB of the same slots.  The block also reduces the chunks' range flags to the unit's flag.
+// Sequential fold of the chunk summaries of one unit and direction, eight key dims per block.  Thread (i, c) owns
+// the four value dims 4 c .. 4 c + 3 of key dim i and takes the chunks in batches of 32, whose loads are all in
+// flight together; the incoming states go out as bf16 tile images.  Every block also reduces the chunks' range
+// flags to the unit's flag.
+constexpr int kFoldRows = 8;
 template <int DV>
-__global__ void __launch_bounds__(32 * (DV / 8))
-bigla_long_fold_kernel(uint8_t* ws_slots, const float* ws_decay, int* ws_flags, const int* ws_cflags, int nch, uint32_t slot_bytes) {
-    constexpr int CPR = DV / 8;   // 16-byte chunks of live value dims per row of the image
-    constexpr int kBatch = 16;
+__global__ void __launch_bounds__(kFoldRows * (DV / 4))
+bigla_long_fold_kernel(const uint8_t* ws_slots, uint8_t* ws_img, const float* ws_decay, int* ws_flags, const int* ws_cflags, int nch,
+                       uint32_t slot_bytes) {
+    constexpr int C4 = DV / 4;   // float4 columns of live value dims
+    constexpr int kBatch = 32;
     const int unit = blockIdx.x, dir = blockIdx.y;
+    const int i = blockIdx.z * kFoldRows + threadIdx.x / C4, c = threadIdx.x % C4;
     pdl_launch_dependents();
     pdl_wait();
     int flagged = 0;
     for (int m = threadIdx.x; m < nch; m += blockDim.x) flagged |= ws_cflags[(size_t)unit * nch + m];
-    flagged = __syncthreads_or(flagged);
-    if (dir == 0 && threadIdx.x == 0) ws_flags[unit] = flagged;
-    if (flagged) return;   // the main launch redoes the unit by the recurrence
-    const int i = threadIdx.x / CPR, c = threadIdx.x % CPR;
-    float carry[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) carry[e] = 0.f;
+    float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int mb = 0; mb < nch; mb += kBatch) {
-        float4 u[kBatch][2];
+        float4 u[kBatch];
         float d[kBatch];
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             if (mb + b < nch) {
                 const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
                 const size_t s = ((size_t)unit * nch + m) * 2 + dir;
-                const float4* src = reinterpret_cast<const float4*>(ws_slots + s * slot_bytes) + ((size_t)i * DV + 8 * c) / 4;
-                u[b][0] = src[0];
-                u[b][1] = src[1];
+                u[b] = *(reinterpret_cast<const float4*>(ws_slots + s * slot_bytes) + ((size_t)i * DV + 4 * c) / 4);
                 d[b] = ws_decay[s * 32 + i];
             }
         }
-        __syncthreads();   // every summary of the batch is in registers before any of its slots is overwritten
+        if (mb == 0) {   // the flags arrive under the latency of the first batch
+            flagged = __syncthreads_or(flagged);
+            if (dir == 0 && blockIdx.z == 0 && threadIdx.x == 0) ws_flags[unit] = flagged;
+        }
+        if (flagged) return;   // the main launch redoes the unit by the recurrence
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             if (mb + b < nch) {
                 const int m = dir == 0 ? mb + b : nch - 1 - (mb + b);
-                uint8_t* img = ws_slots + (((size_t)unit * nch + m) * 2 + dir) * slot_bytes;
+                uint8_t* img = ws_img + (((size_t)unit * nch + m) * 2 + dir) * kImgBytes + i * 128;
                 // forward: the state entering chunk m is the carry; backward: the carry times the chunk's own decay
-                if (dir == 1) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) carry[e] *= d[b];
+                if (dir == 1) { carry.x *= d[b]; carry.y *= d[b]; carry.z *= d[b]; carry.w *= d[b]; }
+                *reinterpret_cast<uint2*>(img + (((c >> 1) ^ (i & 7)) << 4) + (c & 1) * 8) =
+                    make_uint2(pack_bf16(carry.x, carry.y), pack_bf16(carry.z, carry.w));
+                if (c < 16 - C4)   // value dims beyond dv read as zero
+                    *reinterpret_cast<uint2*>(img + ((((C4 + c) >> 1) ^ (i & 7)) << 4) + ((C4 + c) & 1) * 8) = make_uint2(0u, 0u);
+                if (dir == 0) {
+                    carry.x = fmaf(carry.x, d[b], u[b].x); carry.y = fmaf(carry.y, d[b], u[b].y);
+                    carry.z = fmaf(carry.z, d[b], u[b].z); carry.w = fmaf(carry.w, d[b], u[b].w);
+                } else {
+                    carry.x += u[b].x; carry.y += u[b].y; carry.z += u[b].z; carry.w += u[b].w;
                 }
-                uint4 o;
-                o.x = pack_bf16(carry[0], carry[1]); o.y = pack_bf16(carry[2], carry[3]);
-                o.z = pack_bf16(carry[4], carry[5]); o.w = pack_bf16(carry[6], carry[7]);
-                *reinterpret_cast<uint4*>(img + i * 128 + ((c ^ (i & 7)) << 4)) = o;
-                if (c < 8 - CPR)   // value dims beyond dv read as zero
-                    *reinterpret_cast<uint4*>(img + i * 128 + (((CPR + c) ^ (i & 7)) << 4)) = make_uint4(0, 0, 0, 0);
-                const float uu[8] = {u[b][0].x, u[b][0].y, u[b][0].z, u[b][0].w, u[b][1].x, u[b][1].y, u[b][1].z, u[b][1].w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) carry[e] = dir == 0 ? fmaf(carry[e], d[b], uu[e]) : carry[e] + uu[e];
             }
         }
     }
@@ -570,6 +571,7 @@ cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out;
     a.L = L; a.nch = nch; a.tasks = units * nch;
     a.ws_slots = static_cast<uint8_t*>(ws);
+    a.ws_img = static_cast<uint8_t*>(ws) + wl.img_off;
     a.ws_decay = reinterpret_cast<float*>(static_cast<uint8_t*>(ws) + wl.decay_off);
     a.ws_flags = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + wl.flags_off);
     a.ws_cflags = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + wl.cflags_off);
@@ -596,8 +598,8 @@ cudaError_t launch_long_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     const unsigned grid_sum = (unsigned)(a.tasks < cap_sum ? a.tasks : cap_sum), grid_main = (unsigned)(a.tasks < cap_main ? a.tasks : cap_main);
     cudaError_t le = launch_pdl(bigla_long_kernel<DK, DV, kLSummary>, dim3(grid_sum), dim3(kLThreads), smem_sum, stream, tq, tk, tf, tb, tv, to, a);
     if (le == cudaSuccess)
-        le = launch_pdl(bigla_long_fold_kernel<DV>, dim3((unsigned)units, 2), dim3(32 * (DV / 8)), 0, stream, a.ws_slots,
-                        (const float*)a.ws_decay, a.ws_flags, (const int*)a.ws_cflags, nch, a.slot_bytes);
+        le = launch_pdl(bigla_long_fold_kernel<DV>, dim3((unsigned)units, 2, 32 / kFoldRows), dim3(kFoldRows * (DV / 4)), 0, stream,
+                        (const uint8_t*)a.ws_slots, a.ws_img, (const float*)a.ws_decay, a.ws_flags, (const int*)a.ws_cflags, nch, a.slot_bytes);
     if (le == cudaSuccess)
         le = launch_pdl(bigla_long_kernel<DK, DV, kLMain>, dim3(grid_main), dim3(kLThreads), smem_main, stream, tq, tk, tf, tb, tv, to, a);
     if (le != cudaSuccess) return le;
