@@ -32,6 +32,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // batch or a TMA load in flight), then sleeps between polls; gives up after about a quarter of a
 // second and reports it.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+#pragma unroll 1   // many call sites: an unrolled poll loop would multiply the kernels' code size
     for (uint32_t spin = 0; spin < (1u << 21); ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (spin > 4096) __nanosleep(128);
