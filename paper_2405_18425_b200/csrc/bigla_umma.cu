@@ -85,8 +85,7 @@ struct UArgs {
     int* dev_status;
 };
 
-// NC: chunks per unit (1: L <= 128, 2: L <= 256), a template parameter so that either case carries no code of the other.
-template <int DK, int DV, int NC>
+template <int DK, int DV>
 __global__ void __launch_bounds__(kThreads, 2)
 bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_b,
@@ -100,7 +99,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int c = warp >> 2, wq = warp & 3;            // chunk and row quadrant of this warp
     const int L = args.L;
-    constexpr int nc = NC;
+    const int nc = (L + kChunk - 1) / kChunk;
     const int row = c * kChunk + wq * 32 + lane;       // token owned by this thread
     const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
     const bool row_live = row < L;
@@ -609,17 +608,14 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     if (sms == 0) {
         size_t most = make_layout(kMaxRows).total + 1024;
         if (most < rec) most = rec;
-        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
+        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
         if (e != cudaSuccess) return e;
-        if ((e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         sms_of[dev].store(sms, std::memory_order_release);
     }
     // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...
     const long long grid = units < 2LL * sms ? units : 2LL * sms;
-    const cudaError_t le = L <= kChunk
-        ? launch_pdl(bigla_umma_kernel<DK, DV, 1>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a)
-        : launch_pdl(bigla_umma_kernel<DK, DV, 2>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
     count_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
 }
