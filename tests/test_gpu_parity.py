@@ -60,6 +60,18 @@ def test_f32_shapes(oracle, dk, dv, L):
     assert rel_err(got, ref) <= TOL["f32"]
 
 
+@pytest.mark.parametrize("dk,dv", [(32, 64), (24, 48)])
+@pytest.mark.parametrize("L", [127, 128, 129, 130, 144, 145, 208, 255, 256, 257, 258, 384, 385, 513])
+def test_bf16_chunk_boundaries(oracle, dk, dv, L):
+    """Lengths just below, at and just above a multiple of the 128-token chunk: a second (or last) chunk of one
+    or two tokens, the hand-over of the running states across the boundary, the step from the single-block
+    kernel (L <= 256) to the chunk-task kernels; several units per persistent block."""
+    cfg, x = random_problem(700 + L, 5, 3, L, dk, dv, "bf16", gate_mean=1.0)
+    got, ref = _run_unfused(oracle, cfg, x)
+    assert np.isfinite(got).all()
+    assert rel_err(got, ref) <= TOL["bf16"]
+
+
 @pytest.mark.parametrize("L", [600, 2049, 4096 + 37])
 def test_bf16_long_sequences(oracle, L):
     """Sequences split into several segments with a ragged last segment."""
