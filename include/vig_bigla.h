@@ -112,7 +112,7 @@ int vig_bigla_fwd_ws_bf16(const void* q, const void* k, const void* v,
  *     (different streams, no ordering between them) race on it and give undefined results: order them.
  * Results are identical to vig_bigla_fwd_bf16.  Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED,
  * WORKSPACE, CUDA. */
-#define VIG_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+#define VIG_STATIC_SCRATCH_BYTES (24u * 1024u * 1024u)
 int vig_bigla_fwd_static_bf16(const void* q, const void* k, const void* v,
                               const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
                               int B, int H, int L, int dk, int dv, void* stream);

@@ -157,13 +157,18 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
     if (tid == 64 && blockIdx.x < args.tasks) {
         // Warm L2 with this block's first task while the kernel before this one in the stream still runs: a prefetch
-        // consumes nothing, and L2 stays coherent with whatever that kernel is still writing.
+        // consumes nothing, and L2 stays coherent with whatever that kernel is still writing.  The main launch only
+        // asks for q: the summary launch has just read the other tiles, and every prefetch queues in front of the
+        // loads proper in the TMA unit.
         const int pu = (int)(blockIdx.x / nch), pr = (int)(blockIdx.x % nch) * kChunk;
-        tma_prefetch_3d(&tm_k, 0, pr, pu);
-        tma_prefetch_3d(&tm_v, 0, pr, pu);
-        tma_prefetch_3d(&tm_f, 0, pr, pu);
-        tma_prefetch_3d(&tm_b, 0, pr, pu);
-        if (MODE == kLMain) tma_prefetch_3d(&tm_q, 0, pr, pu);
+        if (MODE == kLMain) {
+            tma_prefetch_3d(&tm_q, 0, pr, pu);
+        } else {
+            tma_prefetch_3d(&tm_k, 0, pr, pu);
+            tma_prefetch_3d(&tm_v, 0, pr, pu);
+            tma_prefetch_3d(&tm_f, 0, pr, pu);
+            tma_prefetch_3d(&tm_b, 0, pr, pu);
+        }
     }
     if (tid == 0) {
 #pragma unroll

@@ -9,7 +9,7 @@ namespace {
 
 // Scratch of the no-allocation entry point.  Every GPU whose context loads this library carries
 // these bytes until the process exits, so the size is kept modest: it covers, for example,
-// B*H = 32 sequences of 4096 tokens at dk = 24, dv = 48 (12.8 MB).
+// B*H = 32 sequences of 4096 tokens at dk = 24, dv = 48 (20.3 MiB).
 static __device__ __align__(256) unsigned char g_static_scratch[VIG_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;

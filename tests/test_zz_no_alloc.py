@@ -17,7 +17,7 @@ from helpers import to_device
 
 pytestmark = pytest.mark.gpu
 
-STATIC_BYTES = 16 * 1024 * 1024
+STATIC_BYTES = 24 * 1024 * 1024
 
 
 def _problem(seed, units, L, dk, dv):
