@@ -168,7 +168,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(kTmemCols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
-    build_zero_one_tiles(bp + lay.zf, nullptr, tid);
+    build_zero_one_tile(bp + lay.zf, tid);
     // Tile rows the loads never reach (from `rows` up to the 256-row pitch) are K rows of the prefix-sum product
     // of chunk 1: they must be finite, and nothing but the recurrence scratch ever writes them again.
     auto zero_tail_rows = [&]() {
@@ -256,7 +256,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
 
         if (chunk_on) {
-            // ---- prefix / suffix sums of the log gates (unless they were issued while the previous unit was finishing) ----
+            // ---- prefix sums of the log gates (unless they were issued while the previous unit was finishing) ----
             if (issuer && c == 0 && !(nc == 2 && *early_gates == (int)it)) {
                 wait_bar(bar_g, par);
                 issue_prefix(pair_g);

@@ -183,8 +183,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     // the 240 rows of the 0/1 tile, two passes of 128 threads
-    build_zero_one_tiles(bp + Y::zf, nullptr, tid);
-    build_zero_one_tiles(bp + Y::zf, nullptr, tid + kLThreads);
+    build_zero_one_tile(bp + Y::zf, tid);
+    build_zero_one_tile(bp + Y::zf, tid + kLThreads);
     if (tid < 64) totals[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     fence_async_smem();

@@ -1,5 +1,5 @@
 // Pieces shared by the tcgen05 BiGLA kernels: tcgen05 / TMEM wrappers, shared-memory and instruction
-// descriptors, the 0/1 tiles of the prefix-sum products, masking and packing of the score tile.
+// descriptors, the 0/1 tile of the prefix-sum products, masking and packing of the score tile.
 #pragma once
 #include <cuda.h>
 
@@ -129,7 +129,7 @@ __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) { return ((
 
 constexpr uint32_t kHiK64 = desc_hi(512, 4);     // K-major or MN-major tile with 64-byte rows, 64B swizzle
 constexpr uint32_t kHiV128 = desc_hi(1024, 2);   // MN-major tile with 128-byte rows, 128B swizzle
-constexpr uint32_t kHiZ = desc_hi(256, 0);       // 0/1 tiles, no swizzle
+constexpr uint32_t kHiZ = desc_hi(256, 0);       // 0/1 tile, no swizzle
 
 // 1 / x for a normal, positive x without the special-function unit: a bit-level first guess (within 5.1 %)
 // and Newton steps (one: relative error below 0.26 %, two: below 1e-5).  The result only scales bf16
@@ -143,35 +143,27 @@ __device__ __forceinline__ float fast_rcp(float x) {
 }
 constexpr int kRcpSteps = 1;
 
-// Builds the 240-row 0/1 tiles of the prefix / suffix sums (K-major without swizzle: 8-row groups of 256
-// bytes, each two 8x8 core matrices for K 0..7 and K 8..15).  Rows 0..111 of `zf` are zeros, rows 112..127 the
-// lower triangle (diagonal included), rows 128..239 ones; `zb` (may be null: not built) holds ones, the upper
-// triangle, zeros.  The 128-row window starting at row 112 - 16 j is the operand of K step j.  Threads 0..239
-// of the block write.
-__device__ __forceinline__ void build_zero_one_tiles(uint8_t* zf, uint8_t* zb, int tid) {
+// Builds the 240-row 0/1 tile of the prefix sums (K-major without swizzle: 8-row groups of 256 bytes, each two
+// 8x8 core matrices for K 0..7 and K 8..15).  Rows 0..111 are zeros, rows 112..127 the lower triangle (diagonal
+// included), rows 128..239 ones.  The 128-row window starting at row 112 - 16 j is the operand of K step j.
+// Threads 0..239 of the block write (pass tid + blockDim.x in a second call when the block has fewer).
+__device__ __forceinline__ void build_zero_one_tile(uint8_t* zf, int tid) {
     if (tid < (int)kZRows) {
-        uint32_t f[8], b[8];
+        uint32_t f[8];
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
-            uint32_t wf = 0, wb = 0;
+            uint32_t wf = 0;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int kk = 2 * p + h, u = tid - 112;
                 const bool one_f = tid >= 128 || (tid >= 112 && kk <= u);
-                const bool one_b = tid < 112 || (tid < 128 && kk >= u);
                 wf |= (one_f ? 0x3F80u : 0u) << (16 * h);
-                wb |= (one_b ? 0x3F80u : 0u) << (16 * h);
             }
             f[p] = wf;
-            b[p] = wb;
         }
         const uint32_t off = (uint32_t)(tid >> 3) * 256 + (uint32_t)(tid & 7) * 16;
         *reinterpret_cast<uint4*>(zf + off) = make_uint4(f[0], f[1], f[2], f[3]);
         *reinterpret_cast<uint4*>(zf + off + 128) = make_uint4(f[4], f[5], f[6], f[7]);
-        if (zb) {
-            *reinterpret_cast<uint4*>(zb + off) = make_uint4(b[0], b[1], b[2], b[3]);
-            *reinterpret_cast<uint4*>(zb + off + 128) = make_uint4(b[4], b[5], b[6], b[7]);
-        }
     }
 }
 
