@@ -307,14 +307,15 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             uint32_t qf[4], kf[4], qb[4], kb[4];
 #pragma unroll
                             for (int m = 0; m < 4; ++m) {
-                                // e^{b} on the special-function unit, e^{-b} as its reciprocal on the FMA pipe
+                                // the decaying factors on the special-function unit, the growing ones as their packed reciprocals
                                 const int d0 = 8 * c8 + 2 * m;
                                 const float ex0 = ex2(as_f(pf[hf][d0]) * kLog2e), ex1 = ex2(as_f(pf[hf][d0 + 1]) * kLog2e);
                                 const float ey0 = ex2(as_f(pb[hf][d0]) * kLog2e), ey1 = ex2(as_f(pb[hf][d0 + 1]) * kLog2e);
-                                qf[m] = mul_bf16x2(qv[m], pack_bf16(ex0, ex1));                                              // q~> = q e^{b}
-                                kf[m] = mul_bf16x2(kv[m], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
-                                qb[m] = mul_bf16x2(qv[m], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // q~< = q e^{-x}
-                                kb[m] = mul_bf16x2(kv[m], pack_bf16(ey0, ey1));                                              // k~< = k e^{x}
+                                const uint32_t exp_f = pack_bf16(ex0, ex1), exp_b = pack_bf16(ey0, ey1);
+                                qf[m] = mul_bf16x2(qv[m], exp_f);               // q~> = q e^{b}
+                                kf[m] = mul_bf16x2(kv[m], rcp_bf16x2(exp_f));   // k~> = k e^{-b}
+                                qb[m] = mul_bf16x2(qv[m], rcp_bf16x2(exp_b));   // q~< = q e^{-x}
+                                kb[m] = mul_bf16x2(kv[m], exp_b);               // k~< = k e^{x}
                             }
                             *reinterpret_cast<uint4*>(bp + pair_g + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
                             *reinterpret_cast<uint4*>(bp + pair_qk + lay.tile + off) = make_uint4(kf[0], kf[1], kf[2], kf[3]);

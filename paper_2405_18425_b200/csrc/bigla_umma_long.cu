@@ -279,14 +279,15 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             uint32_t qf[4], qb[4];
 #pragma unroll
                             for (int mm = 0; mm < 4; ++mm) {
-                                // e^{b} on the special-function unit, e^{-b} as its reciprocal on the FMA pipe
+                                // the decaying factors on the special-function unit, the growing ones as their packed reciprocals
                                 const int d0 = 8 * c8 + 2 * mm;
                                 const float ex0 = ex2(as_f(pf[d0]) * kLog2e), ex1 = ex2(as_f(pf[d0 + 1]) * kLog2e);
                                 const float ey0 = ex2(as_f(pb[d0]) * kLog2e), ey1 = ex2(as_f(pb[d0 + 1]) * kLog2e);
-                                qf[mm] = mul_bf16x2(qv[mm], pack_bf16(ex0, ex1));                                              // q~> = q e^{b}
-                                kf[mm] = mul_bf16x2(kv[mm], pack_bf16(fast_rcp<kRcpSteps>(ex0), fast_rcp<kRcpSteps>(ex1)));    // k~> = k e^{-b}
-                                qb[mm] = mul_bf16x2(qv[mm], pack_bf16(fast_rcp<kRcpSteps>(ey0), fast_rcp<kRcpSteps>(ey1)));    // q~< = q e^{-x}
-                                kb[mm] = mul_bf16x2(kv[mm], pack_bf16(ey0, ey1));                                              // k~< = k e^{x}
+                                const uint32_t exp_f = pack_bf16(ex0, ex1), exp_b = pack_bf16(ey0, ey1);
+                                qf[mm] = mul_bf16x2(qv[mm], exp_f);               // q~> = q e^{b}
+                                kf[mm] = mul_bf16x2(kv[mm], rcp_bf16x2(exp_f));   // k~> = k e^{-b}
+                                qb[mm] = mul_bf16x2(qv[mm], rcp_bf16x2(exp_b));   // q~< = q e^{-x}
+                                kb[mm] = mul_bf16x2(kv[mm], exp_b);               // k~< = k e^{x}
                             }
                             *reinterpret_cast<uint4*>(bp + Y::f + off) = make_uint4(qf[0], qf[1], qf[2], qf[3]);
                             *reinterpret_cast<uint4*>(bp + Y::b + off) = make_uint4(qb[0], qb[1], qb[2], qb[3]);
