@@ -112,9 +112,10 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         return;
     }
 
-    const int tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
+    // warp index through a shuffle: uniform for the compiler, so MMA operands derived from it stay in uniform registers
+    const int tid = threadIdx.x, lane = tid & 31, wq = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int L = args.L, nch = args.nch;
-    const bool ctl = tid == 32;   // issues loads, MMAs and stores (warp 1: not a range-check warp)
+    const bool ctl = wq == 1 && lane == 0;   // issues loads, MMAs and stores (warp 1: not a range-check warp)
     // mbarriers: log gates landed, q / k landed, v landed, incoming states landed, MMA batch done
     const uint32_t bar_g = base + Y::misc, bar_qk = bar_g + 8, bar_v = bar_g + 16, bar_s = bar_g + 24, bar_mma = bar_g + 32;
     const uint32_t slot = bar_g + 40;
