@@ -107,9 +107,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
     const bool row_live = row < L;
     const bool chunk_on = c < nc;
-    // One thread per chunk issues that chunk's MMAs; the one of chunk 0 also drives the loads and stores.  They sit in
-    // warps 1 and 5, away from the warps whose first / last rows carry the range checks.
-    const bool issuer = wq == 1 && lane == 0;
+    // One warp per chunk (warps 1 and 5, away from the warps whose first / last rows carry the range checks) issues that
+    // chunk's MMAs, through one elected thread per batch; lane 0 of warp 1 also drives the loads and stores.
+    const bool issue_warp = wq == 1;   // one elected thread of it issues a batch and commits it
     const bool ctl = tid == 32;
     const int ks = chunk_on ? (min(L - c * kChunk, kChunk) + 15) >> 4 : 0;   // 16-token K steps of this chunk
     const int nkeys = ks * 16;
@@ -260,7 +260,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
         if (chunk_on) {
             // ---- prefix sums of the log gates (unless they were issued while the previous unit was finishing) ----
-            if (issuer && c == 0 && !(nc == 2 && *early_gates == (int)it)) {
+            if (issue_warp && c == 0 && !(nc == 2 && *early_gates == (int)it) && elect_one()) {
                 wait_bar(bar_g, par);
                 issue_prefix(pair_g);
             }
@@ -363,7 +363,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             for (int p = 0; p < 2; ++p) {
                 const int n = min(nkeys - 64 * p, 64);   // key columns of this half
                 if (n <= 0) break;
-                if (issuer) {
+                if (issue_warp && elect_one()) {
                     const uint32_t idp = instr_desc(128, n, 0, 0);
 #pragma unroll
                     for (int kk = 0; kk < 2; ++kk) {
@@ -414,7 +414,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
             // ---- chunk summary -> bf16 state tile for the other chunk (two chunks only) ------------------------------
             if (nc == 2) {
-                if (issuer) {
+                if (issue_warp && elect_one()) {
                     wait_bar(bar_v, par);
                     constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
                     const uint32_t ak = desc_lo(t_kb, lay.tile) + row0_64, bv = desc_lo(t_v, 16) + row0_128;
@@ -466,7 +466,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
         if (chunk_on) {
             // ---- out = (P v + q~ S_in) / 2 ------------------------------------------------------------------------
-            if (issuer) {
+            if (issue_warp && elect_one()) {
                 wait_bar(bar_v, par);
                 constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
                 uint32_t acc = 0;
@@ -499,7 +499,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // ... and chunk 0's output has left TMEM block 0, which takes the sums of all four gate blocks
                 named_bar(6, 160);
                 tc_fence_after();
-                if (lane == 0 && *early_gates == (int)it + 1) issue_prefix(pair_qk);
+                if (*early_gates == (int)it + 1 && elect_one()) issue_prefix(pair_qk);
                 __syncwarp();
             }
             if (ctl && has_next) {

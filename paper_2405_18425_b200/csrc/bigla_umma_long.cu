@@ -115,7 +115,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // warp index through a shuffle: uniform for the compiler, so MMA operands derived from it stay in uniform registers
     const int tid = threadIdx.x, lane = tid & 31, wq = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int L = args.L, nch = args.nch;
-    const bool ctl = wq == 1 && lane == 0;   // issues loads, MMAs and stores (warp 1: not a range-check warp)
+    const bool ctl = wq == 1 && lane == 0;   // issues loads and stores (warp 1: not a range-check warp); the MMA batches go out
+                                             // through one elected thread of the same warp
     // mbarriers: log gates landed, q / k landed, v landed, incoming states landed, MMA batch done
     const uint32_t bar_g = base + Y::misc, bar_qk = bar_g + 8, bar_v = bar_g + 16, bar_s = bar_g + 24, bar_mma = bar_g + 32;
     const uint32_t slot = bar_g + 40;
@@ -229,7 +230,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const bool unit_slow = MODE == kLMain && args.ws_flags[unit] != 0;
 
         // ---- prefix sums of both log-gate tiles (side by side along N) -> TMEM columns [0,32) / [32,64) ----------
-        if (ctl) {
+        if (wq == 1 && elect_one()) {
             wait_bar(bar_g, par);
             constexpr uint32_t kIdS = instr_desc(128, 64, 0, 1);
             const uint32_t zf = desc_lo(base + Y::zf, 128);
@@ -323,7 +324,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
         if constexpr (MODE == kLSummary) {
             // ---- U = [k~> | k~<]^T v -> TMEM columns [64,128); rows 0..31: forward, rows 32..63: backward ----------
-            if (ctl) {
+            if (wq == 1 && elect_one()) {
                 wait_bar(bar_v, par);
                 constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
                 const uint32_t ak = desc_lo(t_kf, Y::tile), bv = desc_lo(t_v, 16);   // M blocks: k~>, k~< (then two tiles of no interest)
@@ -369,7 +370,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         for (int p = 0; p < 2; ++p) {
             const int n = min(nkeys - 64 * p, 64);
             if (n <= 0) break;
-            if (ctl) {
+            if (wq == 1 && elect_one()) {
                 const uint32_t idp = instr_desc(128, n, 0, 0);
                 const uint32_t aqf = desc_lo(t_qf, 16), aqb = desc_lo(t_qb, 16), bkf = desc_lo(t_kf, 16), bkb = desc_lo(t_kb, 16);
 #pragma unroll
@@ -421,7 +422,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
 
         // out = (q~> S>_in + q~< S<_in + P v) / 2
-        if (ctl) {
+        if (wq == 1 && elect_one()) {
             wait_bar(bar_v, par);
             wait_bar(bar_s, par);
             constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
