@@ -108,9 +108,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const bool row_live = row < L;
     const bool chunk_on = c < nc;
     // One warp per chunk (warps 1 and 5, away from the warps whose first / last rows carry the range checks) issues that
-    // chunk's MMAs, through one elected thread per batch; lane 0 of warp 1 also drives the loads and stores.
+    // chunk's MMAs, through one elected thread per batch; warp 1 also drives the loads and stores the same way.
     const bool issue_warp = wq == 1;   // one elected thread of it issues a batch and commits it
-    const bool ctl = tid == 32;
+    const bool ctl_warp = warp == 1;   // one elected thread of it drives the loads and stores; the bookkeeping is warp-uniform
     const int ks = chunk_on ? (min(L - c * kChunk, kChunk) + 15) >> 4 : 0;   // 16-token K steps of this chunk
     const int nkeys = ks * 16;
     // mbarriers: log-gate tiles landed, q and k landed, v landed, MMA batches of chunk 0 / chunk 1, prefix sums done
@@ -238,9 +238,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
-    bool v_load_pending = false;      // control thread: the v tile of the current unit has not been requested yet
-    bool next_gates_issued = false;   // control thread: the log gates of the next unit are already on their way
-    bool next_loads_issued = false;   // control thread: so are its q and k
+    bool v_load_pending = false;      // control warp (uniform in it): the v tile of the current unit has not been requested yet
+    bool next_gates_issued = false;   // control warp: the log gates of the next unit are already on their way
+    bool next_loads_issued = false;   // control warp: so are its q and k
     for (long long unit_ll = blockIdx.x; unit_ll < args.units; unit_ll += gridDim.x, ++it) {
         const int unit = (int)unit_ll;
         const uint32_t par = it & 1;
@@ -347,11 +347,13 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const bool any = __any_sync(0xffffffffu, out_of_range);
                 if (lane == 0) slow_slot[c] = any ? 1 : 0;
             }
-            if (ctl && v_load_pending) {
+            if (ctl_warp && v_load_pending) {
                 // The store of the previous unit was issued a phase ago and has read the v tile by now: this
                 // wait is short, and the tile is only needed again when the chunk summaries are formed.
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                load_v(unit);
+                if (elect_one()) {
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    load_v(unit);
+                }
                 v_load_pending = false;
             }
 
@@ -424,15 +426,19 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     umma_commit(bar_mma);
                 }
                 wait_mma();
-                if (ctl && has_next) {
+                if (ctl_warp && has_next) {
                     // The summaries were the last readers of the k~ pair (chunk 1's batch included): the next unit's
                     // log gates go there now, a good two microseconds before they are needed.
-                    wait_bar(bar_mma + 8, (it * (uint32_t)(npass_c1 + 2) + (uint32_t)npass_c1) & 1);
-                    if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
-                        load_gates(unit + (int)gridDim.x, pair_qk);
-                        next_gates_issued = true;
-                        *early_gates = (int)it + 1;   // seen by both issuers after the exchange barrier
+                    bool go = false;
+                    if (elect_one()) {
+                        wait_bar(bar_mma + 8, (it * (uint32_t)(npass_c1 + 2) + (uint32_t)npass_c1) & 1);
+                        go = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0;
+                        if (go) {
+                            load_gates(unit + (int)gridDim.x, pair_qk);
+                            *early_gates = (int)it + 1;   // seen by both issuers after the exchange barrier
+                        }
                     }
+                    if (__any_sync(0xffffffffu, go)) next_gates_issued = true;
                 }
                 if (warp == 1 || warp == 4) {
                     // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
@@ -502,17 +508,20 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (*early_gates == (int)it + 1 && elect_one()) issue_prefix(pair_qk);
                 __syncwarp();
             }
-            if (ctl && has_next) {
+            if (ctl_warp && has_next) {
                 // Every MMA that reads the q~ pair is done once chunk 1's last batch is: the next unit's q and k start
                 // to load under the epilogue and the store (unless this unit must be redone by the recurrence,
                 // whose scratch overlays the tiles).
-                if (nc == 2) wait_bar(bar_mma + 8, ((it + 1) * (uint32_t)(npass_c1 + 2) - 1) & 1);
-                if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
-                    if (!next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
-                    load_qk(unit + (int)gridDim.x, pair_g);
-                    next_gates_issued = true;
-                    next_loads_issued = true;
+                bool go = false;
+                if (elect_one()) {
+                    if (nc == 2) wait_bar(bar_mma + 8, ((it + 1) * (uint32_t)(npass_c1 + 2) - 1) & 1);
+                    go = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0;
+                    if (go) {
+                        if (!next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
+                        load_qk(unit + (int)gridDim.x, pair_g);
+                    }
                 }
+                if (__any_sync(0xffffffffu, go)) next_gates_issued = next_loads_issued = true;
             }
             // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
             if (warp_live) {
@@ -551,11 +560,13 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const bool slow = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) != 0;
         if (timed_out) break;
         if (!slow) {
-            if (ctl) {
-                tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                if (has_next && !next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
-                if (has_next && !next_loads_issued) load_qk(unit + (int)gridDim.x, pair_g);
+            if (ctl_warp) {
+                if (elect_one()) {
+                    tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    if (has_next && !next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
+                    if (has_next && !next_loads_issued) load_qk(unit + (int)gridDim.x, pair_g);
+                }
                 next_gates_issued = next_loads_issued = false;
                 v_load_pending = has_next;   // the v tile only once the store has read it: see above
             }
@@ -569,7 +580,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             zero_tail_rows();
             fence_async_smem();
             __syncthreads();
-            if (ctl && has_next) {
+            if (ctl_warp && has_next && elect_one()) {
                 load_gates(unit + (int)gridDim.x, pair_qk);
                 load_qk(unit + (int)gridDim.x, pair_g);
                 load_v(unit + (int)gridDim.x);
@@ -577,7 +588,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
     }
 
-    if (ctl) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
+    // the last store still reads shared memory (the elected thread is the same every time: it owns the bulk groups)
+    if (ctl_warp && elect_one()) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     // ---- release TMEM (every tcgen05 operation of this block has completed) ----
     tc_fence_before();
     __syncthreads();
