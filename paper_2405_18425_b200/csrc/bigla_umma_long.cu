@@ -115,8 +115,9 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // warp index through a shuffle: uniform for the compiler, so MMA operands derived from it stay in uniform registers
     const int tid = threadIdx.x, lane = tid & 31, wq = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int L = args.L, nch = args.nch;
-    const bool ctl = wq == 1 && lane == 0;   // issues loads and stores (warp 1: not a range-check warp); the MMA batches go out
-                                             // through one elected thread of the same warp
+    // Warp 1 (not a range-check warp) issues the loads, the stores and the MMA batches, each through one elected thread
+    // (always the same one: it owns the bulk-copy groups of the stores); its bookkeeping is warp-uniform.
+    const bool ctl_warp = wq == 1;
     // mbarriers: log gates landed, q / k landed, v landed, incoming states landed, MMA batch done
     const uint32_t bar_g = base + Y::misc, bar_qk = bar_g + 8, bar_v = bar_g + 16, bar_s = bar_g + 24, bar_mma = bar_g + 32;
     const uint32_t slot = bar_g + 40;
@@ -210,13 +211,13 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_after();
     };
 
-    if (ctl && blockIdx.x < args.tasks) {
+    if (ctl_warp && blockIdx.x < args.tasks && elect_one()) {
         load_operands(blockIdx.x);
         load_v(blockIdx.x);
     }
 
     uint32_t it = 0;
-    bool v_load_pending = false;   // control thread: the v tile of the current task has not been requested yet
+    bool v_load_pending = false;   // control warp (uniform in it): the v tile of the current task has not been requested yet
     for (long long task = blockIdx.x; task < args.tasks; task += gridDim.x, ++it) {
         const uint32_t par = it & 1;
         const int unit = task_unit(task), m = task_chunk(task);
@@ -315,10 +316,12 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const bool any = __any_sync(0xffffffffu, out_of_range);
             if (lane == 0) slow_slot[0] = any ? 1 : 0;
         }
-        if (ctl && v_load_pending) {
+        if (ctl_warp && v_load_pending) {
             // the store of the previous task has read the v tile by now; the tile is needed again only further down
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            load_v(task);
+            if (elect_one()) {
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                load_v(task);
+            }
             v_load_pending = false;
         }
 
@@ -334,9 +337,13 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
-            if (ctl && has_next && *time_flag == 0) {   // the summary batch was the last reader of every tile
-                load_operands(next);
-                load_v(next);
+            if (ctl_warp && has_next) {   // the summary batch was the last reader of every tile
+                // (the flag is read into one value for the whole warp first: elect.sync needs all of it)
+                const bool go = __all_sync(0xffffffffu, *time_flag == 0);
+                if (go && elect_one()) {
+                    load_operands(next);
+                    load_v(next);
+                }
             }
             if (wq < 2) {
                 // lane = key dim; warp 0: forward summary, warp 1: backward summary
@@ -381,7 +388,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
-            if (p == 0 && ctl) load_states(task);   // rows 0..63 of k~> and k~< have been read for the last time
+            if (p == 0 && ctl_warp && elect_one()) load_states(task);   // rows 0..63 of k~> and k~< have been read for the last time
             if (warp_live) {
                 uint32_t pk[16];
                 combine_any(2 * p, wq, true, rc, rc + 64, lane, pk);
@@ -439,7 +446,10 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
         wait_mma();
         const bool next_early = has_next && !unit_slow;
-        if (ctl && next_early && *time_flag == 0) load_operands(next);   // every MMA that reads the operand tiles is done
+        if (ctl_warp && next_early) {   // every MMA that reads the operand tiles is done
+            const bool go = __all_sync(0xffffffffu, *time_flag == 0);
+            if (go && elect_one()) load_operands(next);
+        }
         if (warp_live) {
             // epilogue: out = O / 2, bf16, into the dead v tile (same swizzle as the TMA store expects)
 #pragma unroll
@@ -476,10 +486,12 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         handover();
         if (*time_flag != 0) break;
         if (!unit_slow) {
-            if (ctl) {
-                tma_store_3d(&tm_o, 0, m * kChunk, unit, t_v);   // rows >= L and columns >= dv are clipped
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                if (has_next && !next_early) load_operands(next);
+            if (ctl_warp) {
+                if (elect_one()) {
+                    tma_store_3d(&tm_o, 0, m * kChunk, unit, t_v);   // rows >= L and columns >= dv are clipped
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    if (has_next && !next_early) load_operands(next);
+                }
                 v_load_pending = has_next;   // the v tile only once the store has read it
             }
         } else {
@@ -492,7 +504,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 fence_async_smem();
                 __syncthreads();
             }
-            if (ctl && has_next) {
+            if (ctl_warp && has_next && elect_one()) {
                 load_operands(next);
                 load_v(next);
             }
@@ -500,7 +512,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }   // main mode
     }
 
-    if (ctl) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
+    if (ctl_warp && elect_one()) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the last store still reads shared memory
     tc_fence_before();
     __syncthreads();
     if (wq == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kLTmemCols));
