@@ -147,7 +147,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     };
 
     pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
-    if (tid == 64) {
+    if (warp == 2 && elect_one()) {
         // Warm L2 with this block's first unit while the kernel before this one in the stream still runs: a prefetch
         // consumes nothing, and L2 stays coherent with whatever that kernel is still writing.
         tma_prefetch_3d(&tm_q, 0, 0, blockIdx.x);
@@ -185,7 +185,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     zero_tail_rows();
     if (tid < 128) dec[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
-    if (tid == 0) {
+    if (warp == 0 && elect_one()) {
         load_gates(blockIdx.x, 2 * lay.tile);
         load_qk(blockIdx.x, 0);
         load_v(blockIdx.x);
@@ -248,7 +248,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint32_t pair_qk = (it & 1) ? 2 * lay.tile : 0, pair_g = (it & 1) ? 0 : 2 * lay.tile;   // byte offsets of this unit's tile pairs
         const uint32_t t_kb = base + pair_qk, t_kf = t_kb + lay.tile;   // q, k as loaded; k~<, k~> after scaling
         const uint32_t t_qf = base + pair_g, t_qb = t_qf + lay.tile;    // log alpha>, log alpha< as loaded; q~>, q~< after scaling
-        if (tid == 224 && has_next) {
+        if (warp == 7 && has_next && elect_one()) {
             // pull the tiles of this block's next unit into L2
             const int pu = unit + (int)gridDim.x;
             tma_prefetch_3d(&tm_f, 0, 0, pu);
@@ -494,7 +494,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
-            if (tid == 224 && nc == 2 && *early_gates == (int)it + 1) {
+            if (warp == 7 && nc == 2 && *early_gates == (int)it + 1 && elect_one()) {
                 // The packed scores of both chunks have been consumed (this thread has waited for chunk 1's output batch,
                 // now for chunk 0's): their TMEM columns take the next unit's prefix sums, whose log gates have been on
                 // their way since the chunk summaries.  Warp 7 has the fewest rows to write out.

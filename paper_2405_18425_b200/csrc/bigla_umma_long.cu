@@ -158,7 +158,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     };
 
     pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
-    if (tid == 64 && blockIdx.x < args.tasks) {
+    if (wq == 2 && blockIdx.x < args.tasks && elect_one()) {
         // Warm L2 with this block's first task while the kernel before this one in the stream still runs: a prefetch
         // consumes nothing, and L2 stays coherent with whatever that kernel is still writing.  The main launch only
         // asks for q: the summary launch has just read the other tiles, and every prefetch queues in front of the
