@@ -225,12 +225,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint32_t z = desc_lo(base + lay.zf, 128);
         const uint32_t g = desc_lo(base + gates_pair, nc == 2 ? kChunk * 64 : lay.tile);
         const uint32_t ids = instr_desc(128, nc == 2 ? 128 : 64, 0, 1);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (j < ks_c0) {
-                const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                umma_ss(tmem, desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
-            }
+#pragma unroll 1
+        for (int j = 0; j < ks_c0; ++j) {
+            const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+            umma_ss(tmem, desc64(z + win, kHiZ), desc64(g + j * 64, kHiK64), ids, j > 0);
         }
         umma_commit(bar_pfx);
     };
@@ -420,9 +418,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     wait_bar(bar_v, par);
                     constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
                     const uint32_t ak = desc_lo(t_kb, lay.tile) + row0_64, bv = desc_lo(t_v, 16) + row0_128;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        if (kk < ks) umma_ss(tc + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
+#pragma unroll 1   // issue loops stay rolled: less code for the instruction cache, and nothing is gained by unrolling them
+                    for (int kk = 0; kk < ks; ++kk)
+                        umma_ss(tc + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
                     umma_commit(bar_mma);
                 }
                 wait_mma();
@@ -485,12 +483,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     acc = 1;
                 }
                 const uint32_t bv = desc_lo(t_v, 16) + row0_128;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    if (kk < ks) {
-                        umma_ts(tc + 64, tc + kk * 8, desc64(bv + kk * 128, kHiV128), kIdO, kk > 0 ? 1u : acc);
-                    }
-                }
+#pragma unroll 1
+                for (int kk = 0; kk < ks; ++kk) umma_ts(tc + 64, tc + kk * 8, desc64(bv + kk * 128, kHiV128), kIdO, kk > 0 ? 1u : acc);
                 umma_commit(bar_mma);
             }
             wait_mma();

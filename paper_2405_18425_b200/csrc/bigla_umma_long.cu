@@ -236,12 +236,10 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             constexpr uint32_t kIdS = instr_desc(128, 64, 0, 1);
             const uint32_t zf = desc_lo(base + Y::zf, 128);
             const uint32_t g = desc_lo(t_qf, Y::tile);   // second N block: the log alpha< tile
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (j < ks) {
-                    const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
-                    umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(g + j * 64, kHiK64), kIdS, j > 0);
-                }
+#pragma unroll 1   // issue loops stay rolled: less code for the instruction cache
+            for (int j = 0; j < ks; ++j) {
+                const uint32_t win = (uint32_t)(14 - 2 * j) * 16;   // window start row 112 - 16 j
+                umma_ss(tmem + 0, desc64(zf + win, kHiZ), desc64(g + j * 64, kHiK64), kIdS, j > 0);
             }
             umma_commit(bar_mma);
         }
@@ -331,9 +329,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 wait_bar(bar_v, par);
                 constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
                 const uint32_t ak = desc_lo(t_kf, Y::tile), bv = desc_lo(t_v, 16);   // M blocks: k~>, k~< (then two tiles of no interest)
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    if (kk < ks) umma_ss(tmem + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
+#pragma unroll 1
+                for (int kk = 0; kk < ks; ++kk) umma_ss(tmem + 64, desc64(ak + kk * 64, kHiK64), desc64(bv + kk * 128, kHiV128), kIdU, kk > 0);
                 umma_commit(bar_mma);
             }
             wait_mma();
@@ -439,9 +436,8 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             for (int kk = 0; kk < 2; ++kk) umma_ss(tmem + 64, desc64(qf + kk * 2, kHiK64), desc64(sf + kk * 128, kHiV128), kIdO, kk > 0);
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk) umma_ss(tmem + 64, desc64(qb + kk * 2, kHiK64), desc64(sb + kk * 128, kHiV128), kIdO, 1);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-                if (kk < ks) umma_ts(tmem + 64, tmem + kk * 8, desc64(bv + kk * 128, kHiV128), kIdO, 1);
+#pragma unroll 1
+            for (int kk = 0; kk < ks; ++kk) umma_ts(tmem + 64, tmem + kk * 8, desc64(bv + kk * 128, kHiV128), kIdO, 1);
             umma_commit(bar_mma);
         }
         wait_mma();
