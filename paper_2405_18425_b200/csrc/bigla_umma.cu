@@ -538,8 +538,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int ch = 0; ch < DV / 8; ++ch) {
                         uint32_t o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            o[e] = pack_bf16(0.5f * as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e]), 0.5f * as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e + 1]));
+                        for (int e = 0; e < 4; ++e)   // halved after packing: exact (a power of two), one instruction per pair
+                            o[e] = mul_bf16x2(pack_bf16(as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e]), as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e + 1])), 0x3F003F00u);
                         *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }

@@ -458,7 +458,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int ch = 0; ch < 4; ++ch) {
                         uint32_t o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
+                        for (int e = 0; e < 4; ++e) o[e] = mul_bf16x2(pack_bf16(as_f(r[ch * 8 + 2 * e]), as_f(r[ch * 8 + 2 * e + 1])), 0x3F003F00u);   // x 1/2 after packing: exact
                         *reinterpret_cast<uint4*>(bp + Y::v + sw_off<128>(row, hb * 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
@@ -472,7 +472,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int ch = 0; ch < 2; ++ch) {
                         uint32_t o[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) o[e] = pack_bf16(0.5f * as_f(r[ch * 8 + 2 * e]), 0.5f * as_f(r[ch * 8 + 2 * e + 1]));
+                        for (int e = 0; e < 4; ++e) o[e] = mul_bf16x2(pack_bf16(as_f(r[ch * 8 + 2 * e]), as_f(r[ch * 8 + 2 * e + 1])), 0x3F003F00u);   // x 1/2 after packing: exact
                         *reinterpret_cast<uint4*>(bp + Y::v + sw_off<128>(row, 4 + ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
