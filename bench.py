@@ -38,7 +38,7 @@ DEFAULT_WORKLOAD = "vig_b_224"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # captures summarised under profiles/ (None where no capture exists yet).
 NCU_TRAFFIC_BYTES = {
-    "vig_b_224": 59_493_632,    # bigla_umma_kernel<32,64>: 57.88 MB read + 1.62 MB written (profiles/bigla_umma_kernel_vig_b_224.md)
+    "vig_b_224": 59_593_216,    # bigla_umma_kernel<32,64>: 57.87 MB read + 1.72 MB written (profiles/bigla_umma_kernel_vig_b_224.md)
     # vig_t_1024 runs three launches per call; their captures (profiles/bigla_long_kernels_vig_t_1024.md) were taken with
     # flushed caches, which does not describe the L2-resident hand-over between them: no per-call figure is given.
 }
