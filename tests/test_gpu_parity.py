@@ -72,6 +72,36 @@ def test_bf16_chunk_boundaries(oracle, dk, dv, L):
     assert rel_err(got, ref) <= TOL["bf16"]
 
 
+@pytest.mark.parametrize("case", range(24))
+def test_bf16_random_shapes_repeatable(oracle, case):
+    """Seeded random shapes on the tensor-core path (head sizes, lengths on both sides of the 128- and 256-token
+    limits, one to several hundred units, slow and fast gates): parity with the oracle, and the same bits from
+    three back-to-back calls (no result may depend on how the blocks and their pipelines happen to interleave)."""
+    rng = np.random.default_rng(9000 + case)
+    dk, dv = int(rng.choice([16, 24, 32])), int(rng.choice([32, 48, 64]))
+    kind = case % 4
+    L = int(rng.integers(1, 129)) if kind == 0 else int(rng.integers(129, 257)) if kind == 1 else \
+        int(rng.integers(257, 900)) if kind == 2 else int(rng.choice([128, 196, 256, 384, 512]))
+    units = int(rng.integers(1, 40)) if L > 256 else int(rng.integers(1, 700))
+    B = int(rng.integers(1, min(units, 8) + 1))
+    H = max(1, units // B)
+    cfg, x = random_problem(9100 + case, B, H, L, dk, dv, "bf16", gate_mean=float(rng.choice([0.0, 2.0, -1.0, 4.0])))
+    la_f = oracle_log_alpha(oracle, x["g_fwd"], cfg.dtype, cfg.tau)
+    la_b = oracle_log_alpha(oracle, x["g_bwd"], cfg.dtype, cfg.tau)
+    d = {n: to_device(a, cfg.dtype) for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    outs = []
+    for _ in range(3):
+        out = torch.full_like(d["v"], float("nan"))
+        vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], out)
+        outs.append(out)
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    assert all(torch.equal(outs[0].view(torch.int16), o.view(torch.int16)) for o in outs[1:])
+    got = device_to_f64(outs[0], cfg.dtype)
+    assert np.isfinite(got).all()
+    assert rel_err(got, oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, cfg.dtype)) <= TOL["bf16"]
+
+
 @pytest.mark.parametrize("L", [600, 2049, 4096 + 37])
 def test_bf16_long_sequences(oracle, L):
     """Sequences split into several segments with a ragged last segment."""
