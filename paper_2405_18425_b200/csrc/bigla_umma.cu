@@ -209,7 +209,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         ++mma_phase;
         tc_fence_after();
     };
-    // the threads of this chunk have finished their TMEM / shared-memory accesses -> its issuer may go on
+    // the threads of this chunk have finished their TMEM / shared-memory accesses -> its issuing warp may go on
     auto chunk_handover = [&]() {
         tc_fence_before();
         named_bar(1 + c, kChunk);
@@ -433,7 +433,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         go = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0;
                         if (go) {
                             load_gates(unit + (int)gridDim.x, pair_qk);
-                            *early_gates = (int)it + 1;   // seen by both issuers after the exchange barrier
+                            *early_gates = (int)it + 1;   // seen by every warp after the exchange barrier
                         }
                     }
                     if (__any_sync(0xffffffffu, go)) next_gates_issued = true;
