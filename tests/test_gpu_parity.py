@@ -102,6 +102,34 @@ def test_bf16_random_shapes_repeatable(oracle, case):
     assert rel_err(got, oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, cfg.dtype)) <= TOL["bf16"]
 
 
+def test_two_streams_interleaved(oracle):
+    """Calls of different shapes issued alternately on two streams (the long path allocates its scratch per call
+    on the stream it is given): every result equals, bit for bit, the one the same call gives on its own."""
+    problems = []
+    for i, (B, H, L, dk, dv) in enumerate([(3, 4, 196, 32, 64), (1, 3, 1000, 24, 48), (40, 5, 130, 16, 32), (2, 2, 600, 32, 64)]):
+        cfg, x = random_problem(9500 + i, B, H, L, dk, dv, "bf16", gate_mean=1.0)
+        la_f = oracle_log_alpha(oracle, x["g_fwd"], cfg.dtype, cfg.tau)
+        la_b = oracle_log_alpha(oracle, x["g_bwd"], cfg.dtype, cfg.tau)
+        d = {n: to_device(a, cfg.dtype) for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+        alone = torch.empty_like(d["v"])
+        vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], alone)
+        problems.append((d, alone))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    for rep in range(3):
+        for i, (d, _) in enumerate(problems):
+            out = torch.full_like(d["v"], float("nan"))
+            st = streams[(i + rep) % 2]
+            st.wait_stream(torch.cuda.current_stream())
+            vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], out, stream=st)
+            outs.append((i, out))
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    for i, out in outs:
+        assert torch.equal(out.view(torch.int16), problems[i][1].view(torch.int16))
+
+
 @pytest.mark.parametrize("L", [600, 2049, 4096 + 37])
 def test_bf16_long_sequences(oracle, L):
     """Sequences split into several segments with a ragged last segment."""
