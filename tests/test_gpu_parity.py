@@ -102,6 +102,34 @@ def test_bf16_random_shapes_repeatable(oracle, case):
     assert rel_err(got, oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, cfg.dtype)) <= TOL["bf16"]
 
 
+@pytest.mark.parametrize("L", [196, 700])
+def test_cuda_graph_replay(L):
+    """Gate preparation + forward captured into a CUDA graph (the programmatic dependent launches included; the long
+    path with caller-owned scratch, so that nothing allocates during capture) and replayed: same bits as the direct calls."""
+    B, H, dk, dv = 4, 6, 32, 64
+    gen = torch.Generator(device="cuda").manual_seed(77 + L)
+    def mk(d):
+        return torch.randn(B, H, L, d, device="cuda", dtype=torch.bfloat16, generator=gen)
+    q, k, v, gf, gb = mk(dk) * dk ** -0.5, mk(dk), mk(dv), mk(dk) + 1, mk(dk) + 1
+    lf, lb, ref = torch.empty_like(gf), torch.empty_like(gb), torch.empty_like(v)
+    ws = torch.empty(max(vig.vig_bigla_workspace_bytes(B, H, L, dk, dv), 256), dtype=torch.uint8, device="cuda")
+    vig.vig_gate_prep_bf16(gf, gb, lf, lb, 16.0)
+    vig.vig_bigla_fwd_ws_bf16(q, k, v, lf, lb, ref, ws)     # also the first call per device: one-time set-up before capture
+    torch.cuda.synchronize()
+    out = torch.zeros_like(v)
+    s, g = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(g, stream=s):
+            vig.vig_gate_prep_bf16(gf, gb, lf, lb, 16.0, stream=s)
+            vig.vig_bigla_fwd_ws_bf16(q, k, v, lf, lb, out, ws, stream=s)
+    for _ in range(3):
+        out.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert vig.vig_last_device_status() == 0
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+
+
 def test_two_streams_interleaved(oracle):
     """Calls of different shapes issued alternately on two streams (the long path allocates its scratch per call
     on the stream it is given): every result equals, bit for bit, the one the same call gives on its own."""
