@@ -148,20 +148,6 @@ const char* vig_status_string(int status);
  * Returns VIG_OK, VIG_ERR_DEVICE_TIMEOUT if a kernel's bounded wait on an asynchronous copy or on a
  * tensor-core batch expired (the output of that call is then undefined), or VIG_ERR_CUDA. */
 int vig_last_device_status(void* stream);
-/* Which kernel family the bf16 forward entry points use, process-wide (a testing and profiling aid:
- * all families compute the same function and meet the same tolerance).
- *   VIG_KERNEL_AUTO      tcgen05/TMEM kernels for dk in {16,24,32} with dv in {32,48,64} (one persistent
- *                        launch for L <= 256, summary / fold / main launches beyond), else the SIMT
- *                        recurrence                                                       (default)
- *   VIG_KERNEL_MMA_SYNC  the mma.sync tensor-core kernels instead of the tcgen05 ones.  The scratch
- *                        size vig_bigla_workspace_bytes reports depends on this setting: query it
- *                        under the setting the call will run with
- *   VIG_KERNEL_SIMT      always the fp32 SIMT recurrence kernel
- * Returns VIG_OK, or VIG_ERR_UNSUPPORTED for an unknown value (the setting is then unchanged). */
-#define VIG_KERNEL_AUTO 0
-#define VIG_KERNEL_MMA_SYNC 1
-#define VIG_KERNEL_SIMT 2
-int vig_set_kernel_preference(int preference);
 /* Number of kernels this library has launched in this process so far (all devices, all streams). */
 unsigned long long vig_kernel_launch_count(void);
 

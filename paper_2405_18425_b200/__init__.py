@@ -23,8 +23,7 @@ from .binding import (  # noqa: F401
     vig_gate_prep_f32,
     vig_kernel_launch_count,
     vig_last_device_status,
-    vig_set_kernel_preference,
-    VIG_KERNEL_AUTO,
-    VIG_KERNEL_MMA_SYNC,
-    VIG_KERNEL_SIMT,
+    vig_test_set_kernel_preference,
+    VIG_TEST_KERNEL_AUTO,
+    VIG_TEST_KERNEL_SIMT,
 )

@@ -55,8 +55,8 @@ def load() -> ctypes.CDLL:
         lib.vig_status_string.restype = ctypes.c_char_p
         lib.vig_last_device_status.argtypes = [vp]
         lib.vig_last_device_status.restype = ci
-        lib.vig_set_kernel_preference.argtypes = [ci]
-        lib.vig_set_kernel_preference.restype = ci
+        lib.vig_test_set_kernel_preference.argtypes = [ci]
+        lib.vig_test_set_kernel_preference.restype = ci
         lib.vig_kernel_launch_count.argtypes = []
         lib.vig_kernel_launch_count.restype = ctypes.c_ulonglong
         _lib = lib
@@ -176,11 +176,12 @@ def vig_last_device_status(stream=None) -> int:
     return int(load().vig_last_device_status(_stream(stream)))
 
 
-VIG_KERNEL_AUTO, VIG_KERNEL_MMA_SYNC, VIG_KERNEL_SIMT = 0, 1, 2
+VIG_TEST_KERNEL_AUTO, VIG_TEST_KERNEL_SIMT = 0, 2
 
 
-def vig_set_kernel_preference(preference: int) -> None:
-    _check(load().vig_set_kernel_preference(int(preference)), "vig_set_kernel_preference")
+def vig_test_set_kernel_preference(preference: int) -> None:
+    """Test hook (csrc/test_hooks.h; not part of the public C ABI): forces a kernel family process-wide."""
+    _check(load().vig_test_set_kernel_preference(int(preference)), "vig_test_set_kernel_preference")
 
 
 def vig_kernel_launch_count() -> int:

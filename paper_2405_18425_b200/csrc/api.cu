@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cmath>
 
+#include "test_hooks.h"
 #include "vig_internal.h"
 
 namespace vig {
@@ -9,7 +10,7 @@ namespace vig {
 __device__ int g_device_status = 0;
 
 static std::atomic<unsigned long long> g_launches{0};
-static std::atomic<int> g_kernel_pref{VIG_KERNEL_AUTO};
+static std::atomic<int> g_kernel_pref{VIG_TEST_KERNEL_AUTO};   // changed by the test hook only
 int kernel_preference() { return g_kernel_pref.load(std::memory_order_relaxed); }
 void count_launch(unsigned n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -17,6 +18,23 @@ int* device_status_ptr() {
     int* p = nullptr;
     if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status) != cudaSuccess) return nullptr;
     return p;
+}
+
+// ---- dispatch of the bf16 tensor-core path ----------------------------------------------------------------------
+bool tc_supported(int dk, int dv) {
+    return (dk == 16 || dk == 24 || dk == 32) && (dv == 32 || dv == 48 || dv == 64);
+}
+
+size_t tc_workspace_bytes(long long units, int L, int dk, int dv) {
+    if (umma_supported(dk, dv, L)) return 0;   // one thread block covers a unit
+    return umma_long_workspace_bytes(units, L, dk, dv);
+}
+
+cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                            const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
+                            int L, int dk, int dv, void* ws, cudaStream_t stream) {
+    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, stream);
+    return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -43,8 +61,8 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
     const long long units = (long long)B * H;
     using bf = __nv_bfloat16;
     const bf *q_ = (const bf*)q, *k_ = (const bf*)k, *v_ = (const bf*)v, *f_ = (const bf*)la_f, *b_ = (const bf*)la_b;
-    if (mma_supported(dk, dv) && kernel_preference() != VIG_KERNEL_SIMT) {
-        const size_t need = mma_workspace_bytes(units, L, dk, dv);
+    if (tc_supported(dk, dv) && kernel_preference() != VIG_TEST_KERNEL_SIMT) {
+        const size_t need = tc_workspace_bytes(units, L, dk, dv);
         if (!own_ws && need > 0) {
             if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u)) return VIG_ERR_WORKSPACE;
         }
@@ -53,7 +71,7 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
         if (own_ws && need > 0) {
             if (cudaMallocAsync(&scratch, need, stream) != cudaSuccess) return VIG_ERR_CUDA;
         }
-        cudaError_t e = launch_bigla_mma(q_, k_, v_, f_, b_, (bf*)out, units, L, dk, dv, scratch, stream);
+        cudaError_t e = launch_bigla_tc(q_, k_, v_, f_, b_, (bf*)out, units, L, dk, dv, scratch, stream);
         if (own_ws && need > 0) {
             if (cudaFreeAsync(scratch, stream) != cudaSuccess) return VIG_ERR_CUDA;
         }
@@ -122,8 +140,8 @@ int vig_bigla_fwd_f32(const void* q, const void* k, const void* v, const void* l
 
 size_t vig_bigla_workspace_bytes(int B, int H, int L, int dk, int dv, int dtype) {
     if (B <= 0 || H <= 0 || L <= 0 || dk < 1 || dv < 1 || dtype != VIG_DTYPE_BF16) return 0;
-    if (!mma_supported(dk, dv)) return 0;
-    return mma_workspace_bytes((long long)B * H, L, dk, dv);
+    if (!tc_supported(dk, dv)) return 0;
+    return tc_workspace_bytes((long long)B * H, L, dk, dv);
 }
 
 int vig_bigla_fwd_ws_bf16(const void* q, const void* k, const void* v, const void* log_alpha_fwd,
@@ -150,7 +168,7 @@ int vig_bigla_fwd_host(const void* q, const void* k, const void* v, const void* 
     if (!q || !k || !v || !g_fwd || !g_bwd || !out) return VIG_ERR_NULL_POINTER;
     if (B < 0 || H < 0 || L < 0 || dk < 1 || dv < 1 || !(tau > 0.f) || !std::isfinite(tau)) return VIG_ERR_BAD_DIM;
     if (dtype != VIG_DTYPE_F32 && dtype != VIG_DTYPE_BF16) return VIG_ERR_UNSUPPORTED;
-    if (dtype == VIG_DTYPE_F32 ? !recurrence_supported(dk, dv) : !(mma_supported(dk, dv) || recurrence_supported(dk, dv)))
+    if (dtype == VIG_DTYPE_F32 ? !recurrence_supported(dk, dv) : !(tc_supported(dk, dv) || recurrence_supported(dk, dv)))
         return VIG_ERR_UNSUPPORTED;
     if (B == 0 || H == 0 || L == 0) return VIG_OK;
     const size_t es = dtype == VIG_DTYPE_F32 ? 4 : 2;
@@ -209,9 +227,8 @@ int vig_last_device_status(void* stream) {
     return (word & kDevStatusTimeout) ? VIG_ERR_DEVICE_TIMEOUT : VIG_OK;
 }
 
-int vig_set_kernel_preference(int preference) {
-    if (preference != VIG_KERNEL_AUTO && preference != VIG_KERNEL_MMA_SYNC && preference != VIG_KERNEL_SIMT)
-        return VIG_ERR_UNSUPPORTED;
+int vig_test_set_kernel_preference(int preference) {
+    if (preference != VIG_TEST_KERNEL_AUTO && preference != VIG_TEST_KERNEL_SIMT) return VIG_ERR_UNSUPPORTED;
     g_kernel_pref.store(preference, std::memory_order_relaxed);
     return VIG_OK;
 }

@@ -49,16 +49,16 @@ extern "C" int vig_bigla_fwd_static_bf16(const void* q, const void* k, const voi
     const void* ptrs[6] = {q, k, v, log_alpha_fwd, log_alpha_bwd, out};
     for (const void* p : ptrs)
         if (reinterpret_cast<uintptr_t>(p) & 15u) return VIG_ERR_MISALIGNED;
-    if (!mma_supported(dk, dv) || (long long)B * H > 0x7fffffffLL) return VIG_ERR_UNSUPPORTED;
+    if (!tc_supported(dk, dv) || (long long)B * H > 0x7fffffffLL) return VIG_ERR_UNSUPPORTED;
     const long long units = (long long)B * H;
-    const size_t need = mma_workspace_bytes(units, L, dk, dv);
+    const size_t need = tc_workspace_bytes(units, L, dk, dv);
     if (need > (size_t)VIG_STATIC_SCRATCH_BYTES) return VIG_ERR_WORKSPACE;   // beyond the fixed scratch: use the _ws form
     if (B == 0 || H == 0 || L == 0) return VIG_OK;
     void* scratch = nullptr;
     if (static_scratch_ptr(&scratch) != cudaSuccess) return VIG_ERR_CUDA;
-    // Nothing in the scratch has to survive from call to call: the launcher clears the words that must start at
-    // zero on `stream`, and everything else in it is written before it is read within the same call.
-    cudaError_t e = launch_bigla_mma((const bf*)q, (const bf*)k, (const bf*)v, (const bf*)log_alpha_fwd,
+    // Nothing in the scratch has to survive from call to call, and nothing in it has to start at zero: every word
+    // a launch reads to form the result was written earlier in the same call.
+    cudaError_t e = launch_bigla_tc((const bf*)q, (const bf*)k, (const bf*)v, (const bf*)log_alpha_fwd,
                                      (const bf*)log_alpha_bwd, (bf*)out, units, L, dk, dv, scratch,
                                      (cudaStream_t)stream);
     return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;

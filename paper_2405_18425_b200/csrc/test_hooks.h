@@ -1,0 +1,22 @@
+/* Hooks for the library's own tests (exported from libvig_bigla.so, not part of the public C ABI:
+ * include/vig_bigla.h does not declare them and applications must not call them).
+ *
+ * vig_test_set_kernel_preference: which kernel family the bf16 forward entry points use from now on,
+ * process-wide and without any synchronisation against calls in flight on other threads.
+ *   VIG_TEST_KERNEL_AUTO   the default dispatch
+ *   VIG_TEST_KERNEL_SIMT   always the fp32 SIMT recurrence kernel
+ * Returns VIG_OK, or VIG_ERR_UNSUPPORTED for an unknown value (the setting is then unchanged). */
+#ifndef VIG_TEST_HOOKS_H
+#define VIG_TEST_HOOKS_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum vig_test_kernel { VIG_TEST_KERNEL_AUTO = 0, VIG_TEST_KERNEL_SIMT = 2 };
+int vig_test_set_kernel_preference(int preference);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VIG_TEST_HOOKS_H */

@@ -26,13 +26,13 @@ template <typename T>
 cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long long n, float tau,
                              cudaStream_t stream);
 
-// ---- bf16 tensor-core path ----
-bool mma_supported(int dk, int dv);
-// Scratch bytes needed for the segmented (long-L) path; 0 if one thread block covers a unit.
-size_t mma_workspace_bytes(long long units, int L, int dk, int dv);
-cudaError_t launch_bigla_mma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
-                             const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
-                             long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
+// ---- bf16 tensor-core path: dispatch over the tcgen05 kernels (defined with the entry points) ----
+bool tc_supported(int dk, int dv);
+// Scratch bytes the tensor-core path needs for this shape; 0 if no launch of it uses scratch.
+size_t tc_workspace_bytes(long long units, int L, int dk, int dv);
+cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                            const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
+                            long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
 
 // ---- bf16 tcgen05 / TMEM path (units of at most 256 tokens) ----
 bool umma_supported(int dk, int dv, int L);
@@ -64,7 +64,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Kernel family the bf16 entry points prefer (VIG_KERNEL_*), set by vig_set_kernel_preference.
+// Kernel family the bf16 entry points use (a vig_test_kernel value; test_hooks.h): the default unless a test changed it.
 int kernel_preference();
 
 }  // namespace vig

@@ -373,22 +373,22 @@ def test_golden_samples(oracle):
             assert abs(got[t, j] - val) <= TOL[cfg.dtype] * scale
 
 
-@pytest.mark.parametrize("pref", [vig.VIG_KERNEL_AUTO, vig.VIG_KERNEL_MMA_SYNC, vig.VIG_KERNEL_SIMT])
+@pytest.mark.parametrize("pref", [vig.VIG_TEST_KERNEL_AUTO, vig.VIG_TEST_KERNEL_SIMT])
 @pytest.mark.parametrize("dk,dv,L", [(32, 64, 196), (24, 48, 196), (32, 48, 128), (24, 64, 129), (32, 64, 256),
                                      (32, 64, 40), (24, 48, 300)])
 def test_every_kernel_family_meets_the_bar(oracle, pref, dk, dv, L):
-    """The tcgen05 kernel, the mma.sync kernel and the SIMT recurrence kernel behind the same entry point."""
+    """The tcgen05 kernels and the SIMT recurrence kernel behind the same entry point."""
     cfg, x = random_problem(600 + L, 3, 2, L, dk, dv, "bf16")
-    vig.vig_set_kernel_preference(pref)
+    vig.vig_test_set_kernel_preference(pref)
     try:
         got, ref = _run_unfused(oracle, cfg, x)
     finally:
-        vig.vig_set_kernel_preference(vig.VIG_KERNEL_AUTO)
+        vig.vig_test_set_kernel_preference(vig.VIG_TEST_KERNEL_AUTO)
     assert np.isfinite(got).all()
     assert rel_err(got, ref) <= TOL["bf16"]
 
 
 def test_kernel_preference_rejects_unknown_values():
     lib = vig.load()
-    assert lib.vig_set_kernel_preference(7) == -3
-    assert lib.vig_set_kernel_preference(vig.VIG_KERNEL_AUTO) == 0
+    assert lib.vig_test_set_kernel_preference(7) == -3
+    assert lib.vig_test_set_kernel_preference(vig.VIG_TEST_KERNEL_AUTO) == 0
