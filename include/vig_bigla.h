@@ -130,6 +130,20 @@ int vig_gate_prep_f32(const void* g_fwd, const void* g_bwd,
                       void* log_alpha_fwd, void* log_alpha_bwd,
                       int B, int H, int L, int dk, float tau, void* stream);
 
+/* ---- Gate preparation fused into the forward pass (Eq. 5 line 1 / Eq. 6 lines 1-2, then Eq. 6) ------------
+ * out = BiGLA(q, k, v, logsigmoid(g_fwd) / tau, logsigmoid(g_bwd) / tau): the same result contract as
+ * vig_gate_prep_bf16 followed by vig_bigla_fwd_bf16, without the round trip of log alpha through device
+ * memory.  g_fwd, g_bwd: [B,H,L,dk] gate logits (read only); tau > 0.
+ * Units of at most 256 tokens with dk in {16,24,32}, dv in {32,48,64} run in one kernel that turns each gate
+ * tile into log alpha in shared memory (fp32 evaluation with exp and log from the special-function unit,
+ * rounded to bf16 as the tensor-core operand of the prefix sums: the same rounding point as the un-fused
+ * chain).  Longer sequences and other head sizes run gate preparation into scratch the library allocates and
+ * frees on `stream`, then the ordinary forward pass.
+ * Errors: NULL_POINTER, BAD_DIM (also tau), UNSUPPORTED, MISALIGNED, CUDA. */
+int vig_bigla_fwd_gates_bf16(const void* q, const void* k, const void* v,
+                             const void* g_fwd, const void* g_bwd, void* out,
+                             int B, int H, int L, int dk, int dv, float tau, void* stream);
+
 /* ---- Whole path on HOST buffers -------------------------------------------------------------------
  * Gate preparation followed by the BiGLA forward (Eq. 5 line 1 + Eq. 6) for callers whose data
  * lives in host memory.  All seven pointers are HOST pointers (pinned memory makes the copies

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     vig_bigla_fwd,
     vig_bigla_fwd_bf16,
     vig_bigla_fwd_f32,
+    vig_bigla_fwd_gates_bf16,
     vig_bigla_fwd_host,
     vig_bigla_fwd_static_bf16,
     vig_bigla_fwd_ws_bf16,
@@ -26,4 +27,5 @@ from .binding import (  # noqa: F401
     vig_test_set_kernel_preference,
     VIG_TEST_KERNEL_AUTO,
     VIG_TEST_KERNEL_SIMT,
+    VIG_TEST_KERNEL_CHUNK_TASKS,
 )

@@ -49,6 +49,8 @@ def load() -> ctypes.CDLL:
         for name in ("vig_gate_prep_bf16", "vig_gate_prep_f32"):
             getattr(lib, name).argtypes = [vp] * 4 + [ci] * 4 + [cf, vp]
             getattr(lib, name).restype = ci
+        lib.vig_bigla_fwd_gates_bf16.argtypes = [vp] * 6 + [ci] * 5 + [cf, vp]
+        lib.vig_bigla_fwd_gates_bf16.restype = ci
         lib.vig_bigla_fwd_host.argtypes = [vp] * 6 + [ci] * 5 + [cf, ci, vp]
         lib.vig_bigla_fwd_host.restype = ci
         lib.vig_status_string.argtypes = [ci]
@@ -152,6 +154,15 @@ def vig_gate_prep_f32(g_fwd, g_bwd, log_alpha_fwd, log_alpha_bwd, tau=16.0, stre
     return _gate_prep("vig_gate_prep_f32", g_fwd, g_bwd, log_alpha_fwd, log_alpha_bwd, tau, stream)
 
 
+def vig_bigla_fwd_gates_bf16(q, k, v, g_fwd, g_bwd, out, tau=16.0, stream=None):
+    """Forward pass from the gate logits: log alpha = logsigmoid(g) / tau is prepared inside the call."""
+    _dev(q, k, v, g_fwd, g_bwd, out)
+    _check(load().vig_bigla_fwd_gates_bf16(q.data_ptr(), k.data_ptr(), v.data_ptr(), g_fwd.data_ptr(), g_bwd.data_ptr(),
+                                           out.data_ptr(), *_dims(q, v), float(tau), _stream(stream)),
+           "vig_bigla_fwd_gates_bf16")
+    return out
+
+
 def _host_ptr(a) -> int:
     if isinstance(a, torch.Tensor):
         if a.is_cuda or not a.is_contiguous():
@@ -176,7 +187,7 @@ def vig_last_device_status(stream=None) -> int:
     return int(load().vig_last_device_status(_stream(stream)))
 
 
-VIG_TEST_KERNEL_AUTO, VIG_TEST_KERNEL_SIMT = 0, 2
+VIG_TEST_KERNEL_AUTO, VIG_TEST_KERNEL_SIMT, VIG_TEST_KERNEL_CHUNK_TASKS = 0, 2, 3
 
 
 def vig_test_set_kernel_preference(preference: int) -> None:

@@ -25,15 +25,23 @@ bool tc_supported(int dk, int dv) {
     return (dk == 16 || dk == 24 || dk == 32) && (dv == 32 || dv == 48 || dv == 64);
 }
 
+// Sequences of more than 256 tokens: one cooperative launch with a block per 256-token segment (up to 32 segments),
+// the three chunk-task launches beyond that (or when a test asks for them).
+static bool use_segments(int L, int dk, int dv) {
+    return umma_seg_supported(dk, dv, L) && kernel_preference() != VIG_TEST_KERNEL_CHUNK_TASKS;
+}
+
 size_t tc_workspace_bytes(long long units, int L, int dk, int dv) {
     if (umma_supported(dk, dv, L)) return 0;   // one thread block covers a unit
+    if (use_segments(L, dk, dv)) return umma_seg_workspace_bytes(units, L);
     return umma_long_workspace_bytes(units, L, dk, dv);
 }
 
 cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                             const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
                             int L, int dk, int dv, void* ws, cudaStream_t stream) {
-    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, stream);
+    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, 0.f, stream);
+    if (use_segments(L, dk, dv)) return launch_bigla_umma_seg(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
     return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
 }
 
@@ -81,6 +89,34 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
     if (empty) return VIG_OK;
     cudaError_t e = launch_recurrence<bf>(q_, k_, v_, f_, b_, (bf*)out, units, L, dk, dv, stream);
     return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
+// Forward pass from the gate logits (Eq. 5 line 1 + Eq. 6).  Units of at most 256 tokens on the tensor-core shapes:
+// one kernel that prepares log alpha on chip.  Everything else: gate preparation into scratch of the stream, then the
+// ordinary forward pass.
+static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, const void* g_f, const void* g_b, void* out,
+                               int B, int H, int L, int dk, int dv, float tau, cudaStream_t stream) {
+    bool empty;
+    int st = check_fwd_args(q, k, v, g_f, g_b, out, B, H, L, dk, dv, &empty);
+    if (st != VIG_OK) return st;
+    if (!(tau > 0.f) || !std::isfinite(tau)) return VIG_ERR_BAD_DIM;
+    if (!tc_supported(dk, dv) && !recurrence_supported(dk, dv)) return VIG_ERR_UNSUPPORTED;
+    if (empty) return VIG_OK;
+    const long long units = (long long)B * H;
+    using bf = __nv_bfloat16;
+    if (tc_supported(dk, dv) && umma_supported(dk, dv, L) && kernel_preference() == VIG_TEST_KERNEL_AUTO) {
+        cudaError_t e = launch_bigla_umma((const bf*)q, (const bf*)k, (const bf*)v, (const bf*)g_f, (const bf*)g_b, (bf*)out,
+                                          units, L, dk, dv, tau, stream);
+        return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+    }
+    const size_t n = (size_t)units * L * dk;
+    const size_t gate_bytes = (n * sizeof(bf) + 255) / 256 * 256;
+    char* la = nullptr;
+    if (cudaMallocAsync((void**)&la, 2 * gate_bytes, stream) != cudaSuccess) return VIG_ERR_CUDA;
+    st = vig_gate_prep_bf16(g_f, g_b, la, la + gate_bytes, B, H, L, dk, tau, stream);
+    if (st == VIG_OK) st = vig_bigla_fwd_bf16(q, k, v, la, la + gate_bytes, out, B, H, L, dk, dv, stream);
+    if (cudaFreeAsync(la, stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
+    return st;
 }
 
 static int fwd_f32_impl(const void* q, const void* k, const void* v, const void* la_f, const void* la_b, void* out,
@@ -136,6 +172,11 @@ int vig_bigla_fwd(const void* q, const void* k, const void* v, const void* log_a
 int vig_bigla_fwd_f32(const void* q, const void* k, const void* v, const void* log_alpha_fwd,
                       const void* log_alpha_bwd, void* out, int B, int H, int L, int dk, int dv, void* stream) {
     return fwd_f32_impl(q, k, v, log_alpha_fwd, log_alpha_bwd, out, B, H, L, dk, dv, (cudaStream_t)stream);
+}
+
+int vig_bigla_fwd_gates_bf16(const void* q, const void* k, const void* v, const void* g_fwd, const void* g_bwd, void* out,
+                             int B, int H, int L, int dk, int dv, float tau, void* stream) {
+    return fwd_gates_bf16_impl(q, k, v, g_fwd, g_bwd, out, B, H, L, dk, dv, tau, (cudaStream_t)stream);
 }
 
 size_t vig_bigla_workspace_bytes(int B, int H, int L, int dk, int dv, int dtype) {
@@ -228,7 +269,8 @@ int vig_last_device_status(void* stream) {
 }
 
 int vig_test_set_kernel_preference(int preference) {
-    if (preference != VIG_TEST_KERNEL_AUTO && preference != VIG_TEST_KERNEL_SIMT) return VIG_ERR_UNSUPPORTED;
+    if (preference != VIG_TEST_KERNEL_AUTO && preference != VIG_TEST_KERNEL_SIMT && preference != VIG_TEST_KERNEL_CHUNK_TASKS)
+        return VIG_ERR_UNSUPPORTED;
     g_kernel_pref.store(preference, std::memory_order_relaxed);
     return VIG_OK;
 }

@@ -57,21 +57,21 @@ struct ULayout {
                        //   Two chunks: the pitch is 256 rows, so that chunk 0 and chunk 1 of both gate tiles are
                        //   four blocks at one stride, the N blocks of the prefix-sum product.
     uint32_t v;        // v tile [rows][64] bf16 (128B swizzle), later the output tile
-    uint32_t zf;       // 0/1 tile of the prefix sums
     uint32_t s_fwd;    // bf16 state entering chunk 1 from the left  [32][64] (128B swizzle)
-    uint32_t s_bwd;    // bf16 state entering chunk 0 from the right
+    uint32_t s_bwd;    // bf16 state entering chunk 0 from the right  (segmented sequences keep their states elsewhere)
+    uint32_t zf;       // 0/1 tile of the prefix sums
     uint32_t dec;      // [2 chunks][2][32] fp32 totals of the log gates: b and x at the chunk's last row
     uint32_t misc;     // six mbarriers, TMEM slot, flags
     uint32_t total;
 };
-__host__ __device__ inline ULayout make_layout(int rows) {
+__host__ __device__ inline ULayout make_layout(int rows, bool seg) {
     ULayout l;
     l.tile = rows > kChunk ? 2u * kChunk * 64u : (uint32_t)rows * 64u;
     l.v = 4 * l.tile;
-    l.zf = l.v + (uint32_t)rows * 128;
-    l.s_fwd = (l.zf + kZBytes + 1023u) & ~1023u;
-    l.s_bwd = l.s_fwd + 32 * 128;
-    l.dec = l.s_bwd + 32 * 128;
+    l.s_fwd = (l.v + (uint32_t)rows * 128 + 1023u) & ~1023u;
+    l.s_bwd = l.s_fwd + (seg ? 0 : 32 * 128);
+    l.zf = l.s_bwd + (seg ? 0 : 32 * 128);
+    l.dec = l.zf + kZBytes;
     l.misc = l.dec + 4 * 32 * 4;
     l.total = l.misc + 128;
     return l;
@@ -80,28 +80,77 @@ __host__ __device__ inline ULayout make_layout(int rows) {
 struct UArgs {
     const __nv_bfloat16 *q, *k, *v, *la_f, *la_b;
     __nv_bfloat16* out;
-    int L, rows;
+    int L, rows;          // tokens per unit; rows of the TMA boxes (tokens of a block rounded up to 16)
     long long units;
     int* dev_status;
+    // segmented sequences only (SEG): a unit is cut into nseg segments of 256 tokens, one block each
+    int nseg;
+    uint8_t* ws;                  // exchange slots, [units][nseg][kSlotBytes]
+    unsigned long long nonce;     // marks the flags of this call
+    // fused gate preparation only (GATES): la_f / la_b hold the gate logits g, and log alpha = logsigmoid(g) / tau
+    float inv_tau;
 };
 
-template <int DK, int DV>
+// log alpha = logsigmoid(g) / tau (Eq. 5 line 1) for the eight bf16 gate logits of one 16-byte piece, evaluated in
+// fp32 as (min(g, 0) - log(1 + e^{-|g|})) / tau with exp and log from the special-function unit, rounded to bf16.
+__device__ __forceinline__ uint4 log_alpha_piece(uint4 g, float inv_tau) {
+    const float c_log = -0.6931471805599453f * inv_tau;   // log2 -> natural log, over tau, negated
+    uint32_t w[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+        const float2 z = unpack_bf16(w[x]);
+        const float l0 = __log2f(1.f + ex2(-fabsf(z.x) * kLog2e)), l1 = __log2f(1.f + ex2(-fabsf(z.y) * kLog2e));
+        w[x] = pack_bf16(fmaf(l0, c_log, fminf(z.x, 0.f) * inv_tau), fmaf(l1, c_log, fminf(z.y, 0.f) * inv_tau));
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// ---- exchange slot of one (unit, segment) in scratch memory (segmented sequences) -------------------------
+// flag (8 bytes): (nonce << 16) | (out-of-range bit << 15) | number of readers that are done with the slot;
+// then, from byte 256: D>[32], d<[32] (decay of the whole segment per key dim and direction, fp32), from byte 512:
+// E>[32][64] (the forward state a zero input leaves behind the segment) and R[32][64] (what the segment adds to
+// the backward state at its first token), bf16: they only ever feed states that are rounded to bf16 operands.
+constexpr size_t kSlotDecay = 256, kSlotFwd = 512, kSlotBwd = 512 + 32 * 64 * 2, kSlotBytes = 512 + 2 * 32 * 64 * 2;
+constexpr int kMaxSegments = 32;
+
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+template <int DK, int DV, bool SEG, bool GATES>
 __global__ void __launch_bounds__(kThreads, 2)
 bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const UArgs args) {
     static_assert((DK == 16 || DK == 24 || DK == 32) && (DV == 32 || DV == 48 || DV == 64), "unsupported head size");
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* bp = smem_raw + (base - smem_u32(smem_raw));
-    const ULayout lay = make_layout(args.rows);
+    static_assert(!(SEG && GATES), "fused gate preparation is built for the single-block form only");
+    extern __shared__ __align__(1024) uint8_t smem_raw[];   // the swizzled tiles need the 1 KB alignment; no slack is allocated
+    const uint32_t base = smem_u32(smem_raw);
+    uint8_t* bp = smem_raw;
+    if ((base & 1023u) != 0) {   // never expected: reported instead of computing on misplaced tiles
+        if (threadIdx.x == 0) atomicOr(args.dev_status, kDevStatusInternal);
+        return;
+    }
+    const ULayout lay = make_layout(args.rows, SEG);
 
     // The warp index goes through a shuffle so that the compiler knows it, and every address and descriptor derived
     // from it, to be uniform across the warp: the operands of tcgen05.mma then stay in uniform registers instead of
     // being moved there one by one before every MMA (measured: -1 us per call).
     const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int c = warp >> 2, wq = warp & 3;            // chunk and row quadrant of this warp
-    const int L = args.L;
+    // Segmented sequences: block b works on segment b % nseg of the units of group b / nseg; the blocks of a group
+    // take the same units in the same order and exchange their segment summaries through scratch memory.
+    const int nseg = SEG ? args.nseg : 1;
+    const int seg = SEG ? (int)(blockIdx.x % (unsigned)nseg) : 0;
+    const int group = SEG ? (int)(blockIdx.x / (unsigned)nseg) : (int)blockIdx.x;
+    const int ngroups = SEG ? (int)(gridDim.x / (unsigned)nseg) : (int)gridDim.x;
+    const int r0 = seg * kMaxRows;                     // first token of this block's segment
+    const int L = SEG ? min(args.L - r0, kMaxRows) : args.L;   // tokens this block holds
     const int nc = (L + kChunk - 1) / kChunk;
     const int row = c * kChunk + wq * 32 + lane;       // token owned by this thread
     const bool warp_live = c * kChunk + wq * 32 < L;   // the warp holds at least one token
@@ -119,6 +168,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     volatile uint32_t* slot_p = reinterpret_cast<volatile uint32_t*>(bp + lay.misc + 48);
     volatile int* time_flag = reinterpret_cast<volatile int*>(bp + lay.misc + 52);
     volatile int* early_gates = reinterpret_cast<volatile int*>(bp + lay.misc + 72);   // (unit counter + 1) whose next log gates went out early
+    volatile int* unit_slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 76);   // SEG: some segment of the unit left the gate range
     volatile int* slow_slot = reinterpret_cast<volatile int*>(bp + lay.misc + 56);   // [4]: range check per chunk (two used)
     const int ks_c1 = nc == 2 ? (L - kChunk + 15) >> 4 : 0;                          // K steps of chunk 1
     const int npass_c1 = ks_c1 > 4 ? 2 : 1;
@@ -133,28 +183,29 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // finished, and the pair that held the log gates (then q~>, q~<) receives the next (q, k).
     auto load_gates = [&](int unit, uint32_t pair) {
         mbar_expect_tx(bar_g, g_bytes);
-        tma_load_3d(base + pair, &tm_f, 0, 0, unit, bar_g);
-        tma_load_3d(base + pair + lay.tile, &tm_b, 0, -1, unit, bar_g);   // one row low: row 0 takes the zero fill
+        tma_load_3d(base + pair, &tm_f, 0, r0, unit, bar_g);
+        tma_load_3d(base + pair + lay.tile, &tm_b, 0, r0 - 1, unit, bar_g);   // one row low: row 0 takes the token before the
+                                                                              // segment (the zero fill in front of the unit)
     };
     auto load_qk = [&](int unit, uint32_t pair) {
         mbar_expect_tx(bar_qk, g_bytes);
-        tma_load_3d(base + pair, &tm_q, 0, 0, unit, bar_qk);
-        tma_load_3d(base + pair + lay.tile, &tm_k, 0, 0, unit, bar_qk);
+        tma_load_3d(base + pair, &tm_q, 0, r0, unit, bar_qk);
+        tma_load_3d(base + pair + lay.tile, &tm_k, 0, r0, unit, bar_qk);
     };
     auto load_v = [&](int unit) {
         mbar_expect_tx(bar_v, v_bytes);
-        tma_load_3d(t_v, &tm_v, 0, 0, unit, bar_v);
+        tma_load_3d(t_v, &tm_v, 0, r0, unit, bar_v);
     };
 
     pdl_launch_dependents();   // the next kernel's set-up may overlap this grid
     if (warp == 2 && elect_one()) {
         // Warm L2 with this block's first unit while the kernel before this one in the stream still runs: a prefetch
         // consumes nothing, and L2 stays coherent with whatever that kernel is still writing.
-        tma_prefetch_3d(&tm_q, 0, 0, blockIdx.x);
-        tma_prefetch_3d(&tm_k, 0, 0, blockIdx.x);
-        tma_prefetch_3d(&tm_v, 0, 0, blockIdx.x);
-        tma_prefetch_3d(&tm_f, 0, 0, blockIdx.x);
-        tma_prefetch_3d(&tm_b, 0, 0, blockIdx.x);
+        tma_prefetch_3d(&tm_q, 0, r0, group);
+        tma_prefetch_3d(&tm_k, 0, r0, group);
+        tma_prefetch_3d(&tm_v, 0, r0, group);
+        tma_prefetch_3d(&tm_f, 0, r0, group);
+        tma_prefetch_3d(&tm_b, 0, r0, group);
     }
     if (tid == 0) {
 #pragma unroll
@@ -162,6 +213,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(bar_pfx, 1);
         *time_flag = 0;
         *early_gates = -1;
+        *unit_slow_slot = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) slow_slot[i] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -186,9 +238,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid < 128) dec[tid] = 0.f;   // key dims a narrow head never writes
     pdl_wait();   // nothing above touches global memory: it may run while the previous kernel in the stream drains
     if (warp == 0 && elect_one()) {
-        load_gates(blockIdx.x, 2 * lay.tile);
-        load_qk(blockIdx.x, 0);
-        load_v(blockIdx.x);
+        load_gates(group, 2 * lay.tile);
+        load_qk(group, 0);
+        load_v(group);
     }
     fence_async_smem();
     tc_fence_before();
@@ -239,26 +291,45 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     bool v_load_pending = false;      // control warp (uniform in it): the v tile of the current unit has not been requested yet
     bool next_gates_issued = false;   // control warp: the log gates of the next unit are already on their way
     bool next_loads_issued = false;   // control warp: so are its q and k
-    for (long long unit_ll = blockIdx.x; unit_ll < args.units; unit_ll += gridDim.x, ++it) {
+    for (long long unit_ll = group; unit_ll < args.units; unit_ll += ngroups, ++it) {
         const int unit = (int)unit_ll;
         const uint32_t par = it & 1;
-        const bool has_next = unit_ll + gridDim.x < args.units;
+        const bool has_next = unit_ll + ngroups < args.units;
         const uint32_t pair_qk = (it & 1) ? 2 * lay.tile : 0, pair_g = (it & 1) ? 0 : 2 * lay.tile;   // byte offsets of this unit's tile pairs
         const uint32_t t_kb = base + pair_qk, t_kf = t_kb + lay.tile;   // q, k as loaded; k~<, k~> after scaling
         const uint32_t t_qf = base + pair_g, t_qb = t_qf + lay.tile;    // log alpha>, log alpha< as loaded; q~>, q~< after scaling
         if (warp == 7 && has_next && elect_one()) {
             // pull the tiles of this block's next unit into L2
-            const int pu = unit + (int)gridDim.x;
-            tma_prefetch_3d(&tm_f, 0, 0, pu);
-            tma_prefetch_3d(&tm_b, 0, 0, pu);
-            tma_prefetch_3d(&tm_q, 0, 0, pu);
-            tma_prefetch_3d(&tm_k, 0, 0, pu);
-            tma_prefetch_3d(&tm_v, 0, 0, pu);
+            const int pu = unit + ngroups;
+            tma_prefetch_3d(&tm_f, 0, r0, pu);
+            tma_prefetch_3d(&tm_b, 0, r0, pu);
+            tma_prefetch_3d(&tm_q, 0, r0, pu);
+            tma_prefetch_3d(&tm_k, 0, r0, pu);
+            tma_prefetch_3d(&tm_v, 0, r0, pu);
         }
 
+        if constexpr (GATES) {
+            // ---- fused gate preparation: the two gate tiles hold the logits g; thread r rewrites tile row r of both in
+            // place as log alpha.  Rows and columns the loads filled with zeros stay zero (log alpha = 0: no decay, and
+            // k = v = 0 there): the forward tile holds token r in row r, the backward tile token r - 1.
+            wait_bar(bar_g, par);
+            if (tid < args.rows) {
+                const bool f_ok = tid < L, b_ok = tid >= 1 && tid <= L;
+#pragma unroll
+                for (int pc = 0; pc < 4; ++pc) {
+                    if ((pc ^ ((tid >> 1) & 3)) * 8 >= DK) continue;   // this 16-byte piece holds padding columns
+                    uint4* gf = reinterpret_cast<uint4*>(bp + pair_g + (uint32_t)tid * 64 + pc * 16);
+                    uint4* gb = reinterpret_cast<uint4*>(bp + pair_g + lay.tile + (uint32_t)tid * 64 + pc * 16);
+                    if (f_ok) *gf = log_alpha_piece(*gf, args.inv_tau);
+                    if (b_ok) *gb = log_alpha_piece(*gb, args.inv_tau);
+                }
+            }
+            fence_async_smem();
+            __syncthreads();
+        }
         if (chunk_on) {
             // ---- prefix sums of the log gates (unless they were issued while the previous unit was finishing) ----
-            if (issue_warp && c == 0 && !(nc == 2 && *early_gates == (int)it) && elect_one()) {
+            if (issue_warp && c == 0 && (GATES || !(nc == 2 && *early_gates == (int)it)) && elect_one()) {
                 wait_bar(bar_g, par);
                 issue_prefix(pair_g);
             }
@@ -332,7 +403,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             fence_async_smem();   // operand tiles were written through the generic proxy, the MMAs read them through the async proxy
             if (nc == 2 && c == 0) {
                 // the chunk's own hand-over, extended by the arrival of chunk 1's warps (they have read their sums)
-                asm volatile("bar.arrive 5, 160;" ::: "memory");   // chunk 0's totals are written: see the chunk summaries
+                if (!SEG) asm volatile("bar.arrive 5, 160;" ::: "memory");   // chunk 0's totals are written: see the chunk summaries
                 tc_fence_before();
                 named_bar(3, 2 * kChunk);
                 tc_fence_after();
@@ -413,7 +484,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
 
             // ---- chunk summary -> bf16 state tile for the other chunk (two chunks only) ------------------------------
-            if (nc == 2) {
+            if (nc == 2 || SEG) {
                 if (issue_warp && elect_one()) {
                     wait_bar(bar_v, par);
                     constexpr uint32_t kIdU = instr_desc(128, 64, 1, 1);
@@ -424,6 +495,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     umma_commit(bar_mma);
                 }
                 wait_mma();
+            }
+            if (nc == 2 && !SEG) {
                 if (ctl_warp && has_next) {
                     // The summaries were the last readers of the k~ pair (chunk 1's batch included): the next unit's
                     // log gates go there now, a good two microseconds before they are needed.
@@ -432,7 +505,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         wait_bar(bar_mma + 8, (it * (uint32_t)(npass_c1 + 2) + (uint32_t)npass_c1) & 1);
                         go = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0;
                         if (go) {
-                            load_gates(unit + (int)gridDim.x, pair_qk);
+                            load_gates(unit + ngroups, pair_qk);
                             *early_gates = (int)it + 1;   // seen by every warp after the exchange barrier
                         }
                     }
@@ -462,7 +535,182 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             }
         }
-        if (nc == 2) {   // the two chunks exchange their states
+        if (nc == 2 && !SEG) {   // the two chunks exchange their states
+            tc_fence_before();
+            __syncthreads();
+            tc_fence_after();
+        }
+        if constexpr (SEG) {
+            // ---- segmented sequences: summaries of this block's chunks -> segment summary -> exchange with the other
+            // blocks of the unit through scratch memory -> the four incoming states of this block's chunks --------------
+            // With T>(c) = (k~>)^T v and T<(c) = (k~<)^T v of chunk c, D>(c) = e^{b_last(c)}, d<(c) = e^{x_last(c)}:
+            //   forward:  S>_in(c + 1) = D>(c) S>_in(c) + D>(c) T>(c)
+            //   backward: R(c) = T<(c) + d<(c) R(c + 1),  S<_in(c) = d<(c) R(c + 1)   (q~< lacks the chunk's own decay)
+            // and the same two recursions run over the segments with the segment summaries
+            //   D> = D>(0) D>(1), E> = D>(1) D>(0) T>(0) + D>(1) T>(1);   d< = d<(0) d<(1), R = T<(0) + d<(0) T<(1).
+            tc_fence_before();
+            __syncthreads();   // every summary batch of the block is done: the k~ pair is dead
+            tc_fence_after();
+            float* su = reinterpret_cast<float*>(bp + pair_qk);   // [2 chunks][T>, T<][32 key dims][64], 16-byte pieces XORed with the key dim
+            if (chunk_on && wq < 2) {
+                // TMEM lanes 0..31 of the summary hold T<, lanes 32..63 hold T>; lane = key dim
+                float* dst = su + (size_t)((c * 2 + (wq == 1 ? 0 : 1)) * 32 + lane) * 64;
+#pragma unroll
+                for (int hb = 0; hb < 2; ++hb) {
+                    uint32_t r[32];
+                    tmem_ld32(rc + 64 + hb * 32, r);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int x = 0; x < 8; ++x)
+                        reinterpret_cast<uint4*>(dst)[(hb * 8 + x) ^ (lane & 15)] = make_uint4(r[4 * x], r[4 * x + 1], r[4 * x + 2], r[4 * x + 3]);
+                }
+            }
+            __syncthreads();
+            // thread (i, j8): key dim i, value dims 8 j8 .. 8 j8 + 7
+            const int si = tid >> 3, sj = tid & 7;
+            const bool two = nc == 2;
+            const float Df0 = ex2(dec[si] * kLog2e), Db0 = ex2(dec[32 + si] * kLog2e);
+            const float Df1 = two ? ex2(dec[64 + si] * kLog2e) : 1.f, Db1 = two ? ex2(dec[96 + si] * kLog2e) : 1.f;
+            auto su_row = [&](int cc, int dir, float (&o)[8]) {
+                const uint4* src = reinterpret_cast<const uint4*>(su + (size_t)((cc * 2 + dir) * 32 + si) * 64);
+                const uint4 a = src[(2 * sj) ^ (si & 15)], b = src[(2 * sj + 1) ^ (si & 15)];
+                o[0] = as_f(a.x); o[1] = as_f(a.y); o[2] = as_f(a.z); o[3] = as_f(a.w);
+                o[4] = as_f(b.x); o[5] = as_f(b.y); o[6] = as_f(b.z); o[7] = as_f(b.w);
+            };
+            uint8_t* slot_u = args.ws + ((size_t)unit * nseg) * kSlotBytes;   // the unit's slots, one per segment
+            {
+                float tf0[8], tb0[8], tf1[8], tb1[8], e[8], r[8];
+                su_row(0, 0, tf0);
+                su_row(0, 1, tb0);
+                if (two) { su_row(1, 0, tf1); su_row(1, 1, tb1); }
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    if (!two) { tf1[x] = 0.f; tb1[x] = 0.f; }
+                    e[x] = Df1 * (Df0 * tf0[x] + tf1[x]);
+                    r[x] = fmaf(Db0, tb1[x], tb0[x]);
+                }
+                uint8_t* mine = slot_u + (size_t)seg * kSlotBytes;
+                const size_t eoff = (size_t)(si * 64 + sj * 8) * 2;
+                __stcg(reinterpret_cast<uint4*>(mine + kSlotFwd + eoff),
+                       make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])));
+                __stcg(reinterpret_cast<uint4*>(mine + kSlotBwd + eoff),
+                       make_uint4(pack_bf16(r[0], r[1]), pack_bf16(r[2], r[3]), pack_bf16(r[4], r[5]), pack_bf16(r[6], r[7])));
+                if (sj == 0) {
+                    float* dd = reinterpret_cast<float*>(mine + kSlotDecay);
+                    __stcg(dd + si, Df0 * Df1);
+                    __stcg(dd + 32 + si, Db0 * Db1);
+                }
+            }
+            __syncthreads();   // the whole summary is written: the release below, by one thread, publishes all of it
+            if (warp == 0) {
+                const int local_slow = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) != 0;
+                if (lane == 0) {
+                    __threadfence();
+                    st_release_u64(reinterpret_cast<unsigned long long*>(slot_u + (size_t)seg * kSlotBytes),
+                                   (args.nonce << 16) | ((unsigned long long)local_slow << 15));
+                }
+                // lane p waits for the summary of segment p (bounded: the blocks of a group are resident together)
+                bool ok = true;
+                int peer_slow = local_slow;
+                if (lane < nseg && lane != seg) {
+                    const unsigned long long* f = reinterpret_cast<const unsigned long long*>(slot_u + (size_t)lane * kSlotBytes);
+                    ok = false;
+#pragma unroll 1
+                    for (uint32_t spin = 0; spin < (1u << 21); ++spin) {
+                        const unsigned long long v = ld_acquire_u64(f);
+                        if ((v >> 16) == args.nonce) { ok = true; peer_slow = (int)((v >> 15) & 1); break; }
+                        if (spin > 64) __nanosleep(64);
+                    }
+                }
+                const bool all_ok = __all_sync(0xffffffffu, ok);
+                const bool any_slow = __any_sync(0xffffffffu, peer_slow != 0);
+                if (lane == 0) {
+                    if (!all_ok) *time_flag = 1;
+                    *unit_slow_slot = any_slow ? 1 : 0;
+                }
+            }
+            __syncthreads();
+            {
+                // fold the summaries of the segments to the left (forward state entering this segment, ascending) and to
+                // the right (R at the first token of the next segment, descending); up to eight loads per direction are
+                // issued before any of them is used
+                float sin[8], rn[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x) sin[x] = rn[x] = 0.f;
+                const bool usable = *time_flag == 0;   // after a time-out the slots may be incomplete: their values are not used
+                constexpr int kB = 8;
+                const size_t eoff = (size_t)(si * 64 + sj * 8) * 2;
+                int pf = 0, pb = nseg - 1;   // next forward peer (ascending), next backward peer (descending)
+                while (usable && (pf < seg || pb > seg)) {
+                    uint4 ef[kB], rb[kB];
+                    float df[kB], db[kB];
+#pragma unroll
+                    for (int b = 0; b < kB; ++b) {
+                        if (pf + b < seg) {
+                            const uint8_t* sl = slot_u + (size_t)(pf + b) * kSlotBytes;
+                            ef[b] = __ldcg(reinterpret_cast<const uint4*>(sl + kSlotFwd + eoff));
+                            df[b] = __ldcg(reinterpret_cast<const float*>(sl + kSlotDecay) + si);
+                        }
+                        if (pb - b > seg) {
+                            const uint8_t* sl = slot_u + (size_t)(pb - b) * kSlotBytes;
+                            rb[b] = __ldcg(reinterpret_cast<const uint4*>(sl + kSlotBwd + eoff));
+                            db[b] = __ldcg(reinterpret_cast<const float*>(sl + kSlotDecay) + 32 + si);
+                        }
+                    }
+#pragma unroll
+                    for (int b = 0; b < kB; ++b) {
+                        if (pf + b < seg) {
+                            const uint32_t w[4] = {ef[b].x, ef[b].y, ef[b].z, ef[b].w};
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                const float2 t = unpack_bf16(w[x]);
+                                sin[2 * x] = fmaf(df[b], sin[2 * x], t.x);
+                                sin[2 * x + 1] = fmaf(df[b], sin[2 * x + 1], t.y);
+                            }
+                        }
+                        if (pb - b > seg) {
+                            const uint32_t w[4] = {rb[b].x, rb[b].y, rb[b].z, rb[b].w};
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                const float2 t = unpack_bf16(w[x]);
+                                rn[2 * x] = fmaf(db[b], rn[2 * x], t.x);
+                                rn[2 * x + 1] = fmaf(db[b], rn[2 * x + 1], t.y);
+                            }
+                        }
+                    }
+                    pf += kB;
+                    pb -= kB;
+                }
+                // the four incoming states of this block's chunks, as bf16 tiles over the (now dead) summaries
+                float tf0[8], tb1[8];
+                su_row(0, 0, tf0);
+                if (two) su_row(1, 1, tb1);
+                __syncthreads();   // every thread has read what it needs of the summaries
+                uint32_t sf0[4], sf1[4], sb0[4], sb1[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    float f1[2], b1[2], b0[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int y = 2 * x + h;
+                        f1[h] = Df0 * (sin[y] + tf0[y]);                    // S>_in(1) = D>(0) (S>_in(0) + T>(0))
+                        const float r1 = two ? fmaf(Db1, rn[y], tb1[y]) : rn[y];   // R(1)
+                        b1[h] = Db1 * rn[y];                                 // S<_in(1)
+                        b0[h] = Db0 * r1;                                    // S<_in(0)
+                    }
+                    sf0[x] = pack_bf16(sin[2 * x], sin[2 * x + 1]);
+                    sf1[x] = pack_bf16(f1[0], f1[1]);
+                    sb0[x] = pack_bf16(b0[0], b0[1]);
+                    sb1[x] = pack_bf16(b1[0], b1[1]);
+                }
+                uint8_t* st = bp + pair_qk;   // [chunk][S>_in, S<_in] tiles of [32][64] bf16, 128B swizzle
+                const uint32_t so = sw_off<128>(si, sj);
+                *reinterpret_cast<uint4*>(st + 0 * 4096 + so) = make_uint4(sf0[0], sf0[1], sf0[2], sf0[3]);
+                *reinterpret_cast<uint4*>(st + 1 * 4096 + so) = make_uint4(sb0[0], sb0[1], sb0[2], sb0[3]);
+                *reinterpret_cast<uint4*>(st + 2 * 4096 + so) = make_uint4(sf1[0], sf1[1], sf1[2], sf1[3]);
+                *reinterpret_cast<uint4*>(st + 3 * 4096 + so) = make_uint4(sb1[0], sb1[1], sb1[2], sb1[3]);
+                fence_async_smem();
+            }
             tc_fence_before();
             __syncthreads();
             tc_fence_after();
@@ -474,7 +722,16 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 wait_bar(bar_v, par);
                 constexpr uint32_t kIdO = instr_desc(128, 64, 0, 1);
                 uint32_t acc = 0;
-                if (nc == 2) {
+                if constexpr (SEG) {
+                    // both incoming states of this chunk: [chunk][S>_in, S<_in] tiles over the k~ pair
+                    const uint32_t qf = desc_lo(t_qf, 16) + row0_64, qb = desc_lo(t_qb, 16) + row0_64;
+                    const uint32_t sf = desc_lo(base + pair_qk + (uint32_t)c * 8192, 16), sb = sf + (4096 >> 4);
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) umma_ss(tc + 64, desc64(qf + kk * 2, kHiK64), desc64(sf + kk * 128, kHiV128), kIdO, kk > 0);
+#pragma unroll
+                    for (int kk = 0; kk < 2; ++kk) umma_ss(tc + 64, desc64(qb + kk * 2, kHiK64), desc64(sb + kk * 128, kHiV128), kIdO, 1);
+                    acc = 1;
+                } else if (nc == 2) {
                     // chunk 1 receives the forward state of chunk 0, chunk 0 the backward state of chunk 1
                     const uint32_t qa = desc_lo(c == 1 ? t_qf : t_qb, 16) + row0_64;
                     const uint32_t sa = desc_lo(base + (c == 1 ? lay.s_fwd : lay.s_bwd), 16);
@@ -488,7 +745,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
-            if (warp == 7 && nc == 2 && *early_gates == (int)it + 1 && elect_one()) {
+            if (!GATES && warp == 7 && nc == 2 && *early_gates == (int)it + 1 && elect_one()) {
                 // The packed scores of both chunks have been consumed (this thread has waited for chunk 1's output batch,
                 // now for chunk 0's): their TMEM columns take the next unit's prefix sums, whose log gates have been on
                 // their way since the chunk summaries.  Warp 7 has the fewest rows to write out.
@@ -499,7 +756,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 // ... and chunk 0's output has left TMEM block 0, which takes the sums of all four gate blocks
                 named_bar(6, 160);
                 tc_fence_after();
-                if (*early_gates == (int)it + 1 && elect_one()) issue_prefix(pair_qk);
+                if (!GATES && *early_gates == (int)it + 1 && elect_one()) issue_prefix(pair_qk);   // (fused gates: only once they are prepared)
                 __syncwarp();
             }
             if (ctl_warp && has_next) {
@@ -509,10 +766,10 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 bool go = false;
                 if (elect_one()) {
                     if (nc == 2) wait_bar(bar_mma + 8, ((it + 1) * (uint32_t)(npass_c1 + 2) - 1) & 1);
-                    go = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0;
+                    go = (SEG ? *unit_slow_slot : (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3])) == 0 && *time_flag == 0;
                     if (go) {
-                        if (!next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
-                        load_qk(unit + (int)gridDim.x, pair_g);
+                        if (!next_gates_issued) load_gates(unit + ngroups, pair_qk);
+                        load_qk(unit + ngroups, pair_g);
                     }
                 }
                 if (__any_sync(0xffffffffu, go)) next_gates_issued = next_loads_issued = true;
@@ -551,15 +808,23 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         tc_fence_after();
         // every MMA of this unit has completed and every thread has left its tiles: block-uniform decisions
         const bool timed_out = *time_flag != 0;
-        const bool slow = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) != 0;
+        const bool slow = (SEG ? *unit_slow_slot : (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3])) != 0;   // SEG: any segment of the unit
         if (timed_out) break;
+        if (SEG && warp == 7 && lane < nseg && lane != seg) {
+            // This block is done with the other segments' slots of this unit: the last reader of a slot clears its flag, so
+            // that a replay of the same call (a captured graph: same nonce) starts from flags that do not match.  Nothing
+            // waits for this warp before the next unit's first barrier.
+            unsigned long long* f = reinterpret_cast<unsigned long long*>(args.ws + ((size_t)unit * nseg + lane) * kSlotBytes);
+            const unsigned long long old = atomicAdd(f, 1ull);
+            if ((int)(old & 0x7fffull) == nseg - 2) st_release_u64(f, 0ull);
+        }
         if (!slow) {
             if (ctl_warp) {
                 if (elect_one()) {
-                    tma_store_3d(&tm_o, 0, 0, unit, t_v);   // rows >= L and columns >= dv are clipped
+                    tma_store_3d(&tm_o, 0, r0, unit, t_v);   // rows >= L and columns >= dv are clipped
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    if (has_next && !next_gates_issued) load_gates(unit + (int)gridDim.x, pair_qk);
-                    if (has_next && !next_loads_issued) load_qk(unit + (int)gridDim.x, pair_g);
+                    if (has_next && !next_gates_issued) load_gates(unit + ngroups, pair_qk);
+                    if (has_next && !next_loads_issued) load_qk(unit + ngroups, pair_g);
                 }
                 next_gates_issued = next_loads_issued = false;
                 v_load_pending = has_next;   // the v tile only once the store has read it: see above
@@ -567,17 +832,20 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         } else {
             // A gate left the range the factorised tiles can represent: evaluate this unit by the recurrence
             // (its scratch overlays the tiles, so the next loads wait until it is done).
-            const size_t ok = (size_t)unit * L * DK, ov = (size_t)unit * L * DV;
-            recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
-                                           args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));
+            // (segmented sequences: the block of the first segment redoes the whole unit, the others store nothing)
+            if (seg == 0) {
+                const size_t ok = (size_t)unit * args.L * DK, ov = (size_t)unit * args.L * DV;
+                recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
+                                               args.out + ov, args.L, DK, DV, reinterpret_cast<float*>(bp), GATES ? args.inv_tau : 0.f);
+            }
             __syncthreads();
             zero_tail_rows();
             fence_async_smem();
             __syncthreads();
             if (ctl_warp && has_next && elect_one()) {
-                load_gates(unit + (int)gridDim.x, pair_qk);
-                load_qk(unit + (int)gridDim.x, pair_g);
-                load_v(unit + (int)gridDim.x);
+                load_gates(unit + ngroups, pair_qk);
+                load_qk(unit + ngroups, pair_g);
+                load_v(unit + ngroups);
             }
         }
     }
@@ -591,10 +859,44 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0 && *time_flag != 0) atomicOr(args.dev_status, kDevStatusTimeout);
 }
 
-template <int DK, int DV>
+// Resident blocks per SM and SM count of the current device for one instantiation (queried once per device; also
+// opts the kernel in to the shared memory of its longest unit).
+struct DevPlan {
+    int sms, per_sm;
+};
+template <int DK, int DV, bool SEG, bool GATES>
+cudaError_t device_plan(size_t smem_max, DevPlan* out) {
+    static std::atomic<int> sms_of[kMaxDevices], per_sm_of[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    int sms = sms_of[dev].load(std::memory_order_acquire);
+    if (sms == 0) {
+        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV, SEG, GATES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        if (e != cudaSuccess) return e;
+        // Blocks of this kernel an SM holds at once, from the resources themselves: two (2 x 256 of the 512 TMEM columns)
+        // if shared memory (plus the kilobyte the system keeps per block) and the register file admit them.  The occupancy
+        // calculator of the runtime reports one block for this kernel where the hardware runs two.
+        cudaFuncAttributes fa;
+        if ((e = cudaFuncGetAttributes(&fa, bigla_umma_kernel<DK, DV, SEG, GATES>)) != cudaSuccess) return e;
+        int smem_sm = 0, regs_sm = 0;
+        if ((e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev)) != cudaSuccess) return e;
+        const int regs_block = (fa.numRegs + 7) / 8 * 8 * kThreads;
+        const int per_sm = (2 * (smem_max + fa.sharedSizeBytes + 1024) <= (size_t)smem_sm && 2 * regs_block <= regs_sm) ? 2 : 1;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        per_sm_of[dev].store(per_sm, std::memory_order_release);
+        sms_of[dev].store(sms, std::memory_order_release);
+    }
+    out->sms = sms;
+    out->per_sm = per_sm_of[dev].load(std::memory_order_acquire);
+    return cudaSuccess;
+}
+
+// GATES: la_f / la_b are the gate logits and `tau` their temperature (fused gate preparation).
+template <int DK, int DV, bool GATES>
 cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                           const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units, int L,
-                          cudaStream_t stream) {
+                          float tau, cudaStream_t stream) {
     const int rows = (L + 15) / 16 * 16;
     CUtensorMap tq, tk, tf, tb, tv, to;
     if (!make_map(&tq, q, units, L, DK, 32, rows) || !make_map(&tk, k, units, L, DK, 32, rows) ||
@@ -603,29 +905,66 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
         return cudaErrorInvalidValue;
     UArgs a{};
     a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows; a.units = units;
+    a.nseg = 1;
+    a.inv_tau = GATES ? 1.f / tau : 0.f;
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
     // The MMAs of chunk 1 read 128 rows of the operand tiles from row 128 on, i.e. up to (256 - rows) * 64
     // bytes past the last q-type tile: that lands in the v tile, inside the allocation.
-    size_t smem = make_layout(rows).total + 1024;   // slack for the manual 1 KB alignment
-    const size_t rec = (size_t)rec_plan(kThreads, DK, DV).smem_floats * 4 + 1024;
+    size_t smem = make_layout(rows, false).total;
+    const size_t rec = (size_t)rec_plan(kThreads, DK, DV).smem_floats * 4;
     if (smem < rec) smem = rec;
-    // once per device: shared-memory opt-in (for the longest unit the kernel takes) and the SM count
-    static std::atomic<int> sms_of[kMaxDevices];
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    int sms = sms_of[dev].load(std::memory_order_acquire);
-    if (sms == 0) {
-        size_t most = make_layout(kMaxRows).total + 1024;
-        if (most < rec) most = rec;
-        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
-        if (e != cudaSuccess) return e;
-        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-        sms_of[dev].store(sms, std::memory_order_release);
-    }
-    // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...
-    const long long grid = units < 2LL * sms ? units : 2LL * sms;
-    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    size_t most = make_layout(kMaxRows, false).total;
+    if (most < rec) most = rec;
+    DevPlan dp;
+    cudaError_t e = device_plan<DK, DV, false, GATES>(most, &dp);
+    if (e != cudaSuccess) return e;
+    // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...  (Nothing waits for another block
+    // here, so a grid larger than what is resident at once only costs time.)
+    const long long cap = 2LL * dp.sms;
+    const long long grid = units < cap ? units : cap;
+    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV, false, GATES>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    count_launch();
+    return le != cudaSuccess ? le : cudaGetLastError();
+}
+
+// Segmented sequences: a unit of up to kMaxSegments x 256 tokens is cut into segments of 256 tokens, one block each.
+// The blocks of a unit exchange their segment summaries through scratch memory and wait for each other, so the grid
+// is a whole number of groups of nseg blocks and never larger than what the device holds at once: every block is then
+// dispatched without any other block of the grid having to finish first.  (A cooperative launch would have the runtime
+// enforce this, but its occupancy calculator admits only one block of this kernel per SM where the hardware runs two.)
+// Every wait on another block is bounded and ends in VIG_ERR_DEVICE_TIMEOUT should the assumption ever fail.
+std::atomic<unsigned long long> g_seg_calls{0};
+
+template <int DK, int DV>
+cudaError_t launch_umma_seg_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                              const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
+                              int L, void* ws, cudaStream_t stream) {
+    const int nseg = (L + kMaxRows - 1) / kMaxRows;
+    CUtensorMap tq, tk, tf, tb, tv, to;
+    if (!make_map(&tq, q, units, L, DK, 32, kMaxRows) || !make_map(&tk, k, units, L, DK, 32, kMaxRows) ||
+        !make_map(&tf, la_f, units, L, DK, 32, kMaxRows) || !make_map(&tb, la_b, units, L, DK, 32, kMaxRows) ||
+        !make_map(&tv, v, units, L, DV, 64, kMaxRows) || !make_map(&to, out, units, L, DV, 64, kMaxRows))
+        return cudaErrorInvalidValue;
+    UArgs a{};
+    a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = kMaxRows; a.units = units;
+    a.nseg = nseg;
+    a.ws = static_cast<uint8_t*>(ws);
+    // the flags of this call: a value no earlier call wrote and no uninitialised word holds by chance (48 bits)
+    a.nonce = (0x5A17ull << 32) + (g_seg_calls.fetch_add(1, std::memory_order_relaxed) & 0xffffffffull) + 1;
+    a.dev_status = device_status_ptr();
+    if (!a.dev_status) return cudaErrorUnknown;
+    size_t smem = make_layout(kMaxRows, true).total;
+    const size_t rec = (size_t)rec_plan(kThreads, DK, DV).smem_floats * 4;
+    if (smem < rec) smem = rec;
+    DevPlan dp;
+    cudaError_t e = device_plan<DK, DV, true, false>(smem, &dp);
+    if (e != cudaSuccess) return e;
+    const long long cap = (long long)dp.per_sm * dp.sms;
+    long long groups = cap / nseg;
+    if (groups < 1) return cudaErrorLaunchOutOfResources;
+    if (groups > units) groups = units;
+    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV, true, false>, dim3((unsigned)(groups * nseg)), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
     count_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
 }
@@ -636,11 +975,34 @@ bool umma_supported(int dk, int dv, int L) {
     return (dk == 16 || dk == 24 || dk == 32) && (dv == 32 || dv == 48 || dv == 64) && L <= kMaxRows;
 }
 
+bool umma_seg_supported(int dk, int dv, int L) {
+    return (dk == 16 || dk == 24 || dk == 32) && (dv == 32 || dv == 48 || dv == 64) && L > kMaxRows &&
+           L <= kMaxSegments * kMaxRows;
+}
+
+size_t umma_seg_workspace_bytes(long long units, int L) {
+    return (size_t)units * (size_t)((L + kMaxRows - 1) / kMaxRows) * kSlotBytes;
+}
+
+cudaError_t launch_bigla_umma_seg(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                  const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
+                                  int L, int dk, int dv, void* ws, cudaStream_t stream) {
+#define VIG_CASE(DK_, DV_) \
+    if (dk == DK_ && dv == DV_) return launch_umma_seg_t<DK_, DV_>(q, k, v, la_f, la_b, out, units, L, ws, stream);
+    VIG_CASE(16, 32) VIG_CASE(16, 48) VIG_CASE(16, 64)
+    VIG_CASE(24, 32) VIG_CASE(24, 48) VIG_CASE(24, 64)
+    VIG_CASE(32, 32) VIG_CASE(32, 48) VIG_CASE(32, 64)
+#undef VIG_CASE
+    return cudaErrorNotSupported;
+}
+
 cudaError_t launch_bigla_umma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                               const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
-                              int L, int dk, int dv, cudaStream_t stream) {
-#define VIG_CASE(DK_, DV_) \
-    if (dk == DK_ && dv == DV_) return launch_umma_t<DK_, DV_>(q, k, v, la_f, la_b, out, units, L, stream);
+                              int L, int dk, int dv, float gate_tau, cudaStream_t stream) {
+#define VIG_CASE(DK_, DV_)                                                                                              \
+    if (dk == DK_ && dv == DV_)                                                                                         \
+        return gate_tau > 0.f ? launch_umma_t<DK_, DV_, true>(q, k, v, la_f, la_b, out, units, L, gate_tau, stream)     \
+                              : launch_umma_t<DK_, DV_, false>(q, k, v, la_f, la_b, out, units, L, 0.f, stream);
     VIG_CASE(16, 32) VIG_CASE(16, 48) VIG_CASE(16, 64)
     VIG_CASE(24, 32) VIG_CASE(24, 48) VIG_CASE(24, 64)
     VIG_CASE(32, 32) VIG_CASE(32, 48) VIG_CASE(32, 64)

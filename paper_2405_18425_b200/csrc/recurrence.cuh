@@ -38,10 +38,11 @@ __device__ __forceinline__ void rec_store(__nv_bfloat16* p, float x) { *p = __fl
 // All threads of the block must call this (it uses __syncthreads).  q, k, la_f, la_b: [L, dk];
 // v, out: [L, dv] of this unit (global or shared memory); ws: rec_plan(...).smem_floats floats of
 // shared memory.  The forward pass stores o> in `out` (rounded to T), the backward pass turns it
-// into (o> + o<)/2.
+// into (o> + o<)/2.  gate_inv_tau > 0: la_f / la_b hold gate logits g instead, and log alpha = logsigmoid(g) / tau
+// (Eq. 5 line 1) is taken on the fly.
 template <typename T>
 __device__ void recurrence_unit(const T* q, const T* k, const T* v, const T* la_f, const T* la_b, T* out,
-                                int L, int dk, int dv, float* ws) {
+                                int L, int dk, int dv, float* ws, float gate_inv_tau = 0.f) {
     const int nt = blockDim.x, tid = threadIdx.x;
     const RecPlan pl = rec_plan(nt, dk, dv);
     float* qs = ws;
@@ -69,7 +70,9 @@ __device__ void recurrence_unit(const T* q, const T* k, const T* v, const T* la_
                 const size_t g = (size_t)t0 * dk + x;
                 qs[x] = rec_to_float(q[g]);
                 ks[x] = rec_to_float(k[g]);
-                es[x] = expf(rec_to_float(la[g]));   // alpha_t[i]
+                float a = rec_to_float(la[g]);
+                if (gate_inv_tau > 0.f) a = (fminf(a, 0.f) - log1pf(expf(-fabsf(a)))) * gate_inv_tau;
+                es[x] = expf(a);   // alpha_t[i]
             }
             for (int x = tid; x < nv * dv; x += nt) vs[x] = rec_to_float(v[(size_t)t0 * dv + x]);
             __syncthreads();

@@ -36,9 +36,18 @@ cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, cons
 
 // ---- bf16 tcgen05 / TMEM path (units of at most 256 tokens) ----
 bool umma_supported(int dk, int dv, int L);
+// gate_tau > 0: la_f / la_b hold the gate logits g and the kernel prepares log alpha = logsigmoid(g) / gate_tau itself.
 cudaError_t launch_bigla_umma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                               const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
-                              long long units, int L, int dk, int dv, cudaStream_t stream);
+                              long long units, int L, int dk, int dv, float gate_tau, cudaStream_t stream);
+
+// ---- the same kernel for sequences of up to 32 x 256 tokens: one block per 256-token segment, the blocks of a unit
+// exchange their segment summaries through scratch memory inside one cooperative launch ----
+bool umma_seg_supported(int dk, int dv, int L);
+size_t umma_seg_workspace_bytes(long long units, int L);
+cudaError_t launch_bigla_umma_seg(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
+                                  const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
+                                  long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
 
 // ---- bf16 tcgen05 / TMEM path for longer sequences: chunk tasks, states through scratch (three launches) ----
 size_t umma_long_workspace_bytes(long long units, int L, int dk, int dv);

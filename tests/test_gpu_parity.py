@@ -10,7 +10,7 @@ import torch
 import paper_2405_18425_b200 as vig
 from paper_2405_18425_b200 import synth
 
-from helpers import (TOL, device_to_f64, oracle_log_alpha, oracle_out, random_problem, rel_err, to_device,
+from helpers import (NTHREADS, TOL, device_to_f64, oracle_log_alpha, oracle_out, random_problem, rel_err, to_device,
                      to_stored)
 
 pytestmark = pytest.mark.gpu
@@ -158,15 +158,54 @@ def test_two_streams_interleaved(oracle):
         assert torch.equal(out.view(torch.int16), problems[i][1].view(torch.int16))
 
 
-@pytest.mark.parametrize("L", [600, 2049, 4096 + 37])
-def test_bf16_long_sequences(oracle, L):
-    """Sequences split into several segments with a ragged last segment."""
+@pytest.fixture
+def chunk_task_path():
+    """Sequences of more than 256 tokens on the three chunk-task launches instead of the segmented launch."""
+    vig.vig_test_set_kernel_preference(vig.VIG_TEST_KERNEL_CHUNK_TASKS)
+    yield
+    vig.vig_test_set_kernel_preference(vig.VIG_TEST_KERNEL_AUTO)
+
+
+def _long_sequences(oracle, L):
     cfg, x = random_problem(300 + L, 1, 3, L, 24, 48, "bf16")
     got, ref = _run_unfused(oracle, cfg, x)
     assert rel_err(got, ref) <= TOL["bf16"]
     cfg, x = random_problem(301 + L, 1, 2, L, 32, 64, "bf16", gate_mean=2.0)
     got, ref = _run_unfused(oracle, cfg, x)
     assert rel_err(got, ref) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("L", [600, 2049, 4096 + 37, 8192, 8192 + 5, 16384])
+def test_bf16_long_sequences(oracle, L):
+    """Sequences split into several segments with a ragged last segment: one block per 256-token segment inside one
+    launch up to 8192 tokens, chunk tasks over three launches beyond."""
+    _long_sequences(oracle, L)
+
+
+@pytest.mark.parametrize("L", [300, 600, 2049, 4096 + 37])
+def test_bf16_long_sequences_chunk_tasks(oracle, chunk_task_path, L):
+    _long_sequences(oracle, L)
+
+
+@pytest.mark.parametrize("units,L", [(1, 257), (3, 384), (40, 513), (700, 300), (5, 8000), (37, 4096)])
+def test_bf16_segmented_groups(oracle, units, L):
+    """The segmented launch with fewer units than groups, more units than groups (several rounds per block), a
+    one-token last segment and the longest sequences; three calls must give the same bits."""
+    cfg, x = random_problem(1300 + L, units, 1, L, 24, 48, "bf16", gate_mean=1.0)
+    la_f = oracle_log_alpha(oracle, x["g_fwd"], cfg.dtype, cfg.tau)
+    la_b = oracle_log_alpha(oracle, x["g_bwd"], cfg.dtype, cfg.tau)
+    d = {n: to_device(a, cfg.dtype) for n, a in dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b).items()}
+    outs = []
+    for _ in range(3):
+        out = torch.full_like(d["v"], float("nan"))
+        vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], d["f"], d["b"], out)
+        outs.append(out)
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    assert all(torch.equal(outs[0].view(torch.int16), o.view(torch.int16)) for o in outs[1:])
+    got = device_to_f64(outs[0], cfg.dtype)
+    assert np.isfinite(got).all()
+    assert rel_err(got, oracle_out(oracle, x["q"], x["k"], x["v"], la_f, la_b, cfg.dtype)) <= TOL["bf16"]
 
 
 def _gate_cases(L, dk, rng):
@@ -265,6 +304,77 @@ def test_whole_path_gate_prep_then_forward(oracle):
     ref = oracle.bigla_fwd(f("q"), f("k"), f("v"), oracle.gate_prep(f("g_fwd"), cfg.tau),
                            oracle.gate_prep(f("g_bwd"), cfg.tau), nthreads=8)
     assert rel_err(device_to_f64(out, cfg.dtype), ref) <= TOL["bf16"]
+
+
+def _run_fused(oracle, cfg, x, tau=None):
+    """GPU forward from the gate logits against the oracle chain gate_prep -> bigla_fwd with fp64 gates in between."""
+    tau = cfg.tau if tau is None else tau
+    d = {n: to_device(a, cfg.dtype) for n, a in x.items()}
+    out = torch.full_like(d["v"], float("nan"))
+    vig.vig_bigla_fwd_gates_bf16(d["q"], d["k"], d["v"], d["g_fwd"], d["g_bwd"], out, tau)
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    f = lambda n: synth.stored_to_f64(x[n], cfg.dtype)
+    ref = oracle.bigla_fwd(f("q"), f("k"), f("v"), oracle.gate_prep(f("g_fwd"), tau), oracle.gate_prep(f("g_bwd"), tau),
+                           nthreads=NTHREADS)
+    for n in x:   # inputs are never written
+        np.testing.assert_array_equal(to_stored(d[n], cfg.dtype), x[n])
+    return device_to_f64(out, cfg.dtype), ref
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4], ids=[c.name for c in synth.CONFIGS[1:]])
+def test_fused_gates_full_size(oracle, idx):
+    """Eq. 5 line 1 + Eq. 6 in one call on the four bf16 configurations at full size, every element compared."""
+    cfg = synth.CONFIGS[idx]
+    got, ref = _run_fused(oracle, cfg, synth.make_inputs(cfg))
+    assert np.isfinite(got).all()
+    err = rel_err(got, ref)
+    print(f"fused gates {cfg.name}: max|gpu-oracle|/max|oracle| = {err:.3e}")
+    assert err <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("dk,dv", [(16, 32), (24, 48), (32, 64), (24, 64), (40, 72)])
+@pytest.mark.parametrize("L", [1, 5, 16, 17, 100, 128, 129, 196, 250, 255, 256, 300])
+def test_fused_gates_small_and_ragged(oracle, dk, dv, L):
+    """Ragged lengths on both sides of the chunk boundary (the padded rows and columns of the gate tiles must stay
+    out of the sums), the last shape off the tensor-core set, L = 300 through gate preparation into scratch."""
+    cfg, x = random_problem(2100 + L, 3, 2, L, dk, dv, "bf16", gate_mean=1.0)
+    got, ref = _run_fused(oracle, cfg, x)
+    assert np.isfinite(got).all()
+    assert rel_err(got, ref) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("tau", [1.0, 3.0, 16.0, 64.0])
+def test_fused_gates_temperature_and_extreme_logits(oracle, tau):
+    """tau = 1 makes the gates steep (padded columns must not trip the range check), tau = 64 nearly open; logits
+    of +-50 and -200 reach both asymptotes of logsigmoid, the last ones through the in-kernel recurrence."""
+    cfg, x = random_problem(2300, 2, 3, 196, 24, 48, "bf16", gate_mean=2.0, tau=tau)
+    got, ref = _run_fused(oracle, cfg, x)
+    assert rel_err(got, ref) <= TOL["bf16"]
+    g = synth.stored_to_f64(x["g_fwd"], "bf16").copy()
+    g[0, 1, 30:34] = 50.0
+    g[1, 0, 100:103] = -50.0
+    g[1, 2, 7] = -200.0
+    x2 = dict(x, g_fwd=synth.store(g, "bf16"), g_bwd=synth.store(g[:, :, ::-1].copy(), "bf16"))
+    got, ref = _run_fused(oracle, cfg, x2, tau)
+    assert np.isfinite(got).all()
+    assert rel_err(got, ref) <= TOL["bf16"]
+
+
+def test_fused_gates_match_unfused_chain_closely():
+    """The fused kernel rounds log alpha to bf16 at the same point as the un-fused chain, so the two GPU results agree
+    far inside the tolerance (not bit for bit: the special-function unit stands in for log1p)."""
+    cfg = synth.CONFIGS[3]
+    x = synth.make_inputs(cfg, units=slice(0, 48))
+    d = {n: to_device(a, cfg.dtype) for n, a in x.items()}
+    la_f, la_b = torch.empty_like(d["g_fwd"]), torch.empty_like(d["g_bwd"])
+    vig.vig_gate_prep_bf16(d["g_fwd"], d["g_bwd"], la_f, la_b, cfg.tau)
+    a, b = torch.empty_like(d["v"]), torch.empty_like(d["v"])
+    vig.vig_bigla_fwd_bf16(d["q"], d["k"], d["v"], la_f, la_b, a)
+    vig.vig_bigla_fwd_gates_bf16(d["q"], d["k"], d["v"], d["g_fwd"], d["g_bwd"], b, cfg.tau)
+    torch.cuda.synchronize()
+    fa, fb = device_to_f64(a, "bf16"), device_to_f64(b, "bf16")
+    assert np.abs(fa - fb).max() <= 4e-3 * np.abs(fa).max()
 
 
 @pytest.mark.parametrize("idx", [0, 3, 4])
@@ -373,7 +483,7 @@ def test_golden_samples(oracle):
             assert abs(got[t, j] - val) <= TOL[cfg.dtype] * scale
 
 
-@pytest.mark.parametrize("pref", [vig.VIG_TEST_KERNEL_AUTO, vig.VIG_TEST_KERNEL_SIMT])
+@pytest.mark.parametrize("pref", [vig.VIG_TEST_KERNEL_AUTO, vig.VIG_TEST_KERNEL_SIMT, vig.VIG_TEST_KERNEL_CHUNK_TASKS])
 @pytest.mark.parametrize("dk,dv,L", [(32, 64, 196), (24, 48, 196), (32, 48, 128), (24, 64, 129), (32, 64, 256),
                                      (32, 64, 40), (24, 48, 300)])
 def test_every_kernel_family_meets_the_bar(oracle, pref, dk, dv, L):
