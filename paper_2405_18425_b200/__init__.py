@@ -28,4 +28,5 @@ from .binding import (  # noqa: F401
     VIG_TEST_KERNEL_AUTO,
     VIG_TEST_KERNEL_SIMT,
     VIG_TEST_KERNEL_CHUNK_TASKS,
+    VIG_TEST_KERNEL_SEGMENTS,
 )

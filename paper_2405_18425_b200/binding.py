@@ -187,7 +187,7 @@ def vig_last_device_status(stream=None) -> int:
     return int(load().vig_last_device_status(_stream(stream)))
 
 
-VIG_TEST_KERNEL_AUTO, VIG_TEST_KERNEL_SIMT, VIG_TEST_KERNEL_CHUNK_TASKS = 0, 2, 3
+VIG_TEST_KERNEL_AUTO, VIG_TEST_KERNEL_SIMT, VIG_TEST_KERNEL_CHUNK_TASKS, VIG_TEST_KERNEL_SEGMENTS = 0, 2, 3, 4
 
 
 def vig_test_set_kernel_preference(preference: int) -> None:

@@ -25,15 +25,31 @@ bool tc_supported(int dk, int dv) {
     return (dk == 16 || dk == 24 || dk == 32) && (dv == 32 || dv == 48 || dv == 64);
 }
 
-// Sequences of more than 256 tokens: one cooperative launch with a block per 256-token segment (up to 32 segments),
-// the three chunk-task launches beyond that (or when a test asks for them).
-static bool use_segments(int L, int dk, int dv) {
-    return umma_seg_supported(dk, dv, L) && kernel_preference() != VIG_TEST_KERNEL_CHUNK_TASKS;
+// Sequences of more than 256 tokens.  One launch with a block per 256-token segment reads every input once, but the
+// blocks of a unit stall together while they exchange their summaries, and every block reads every other segment's
+// summary: measured against the three chunk-task launches it wins for two segments, and for up to eight when all
+// units are resident at once (one round); the chunk tasks take the rest.  Tests can force either.
+static bool use_segments(long long units, int L, int dk, int dv) {
+    if (!umma_seg_supported(dk, dv, L)) return false;
+    const int pref = kernel_preference();
+    if (pref == VIG_TEST_KERNEL_CHUNK_TASKS) return false;
+    if (pref == VIG_TEST_KERNEL_SEGMENTS) return true;
+    const int nseg = (L + 255) / 256;
+    if (nseg <= 2) return true;
+    if (nseg > 8) return false;
+    static std::atomic<int> sms_cached{0};
+    int sms = sms_cached.load(std::memory_order_relaxed);
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+        sms_cached.store(sms, std::memory_order_relaxed);
+    }
+    return units * nseg <= 2LL * sms;
 }
 
 size_t tc_workspace_bytes(long long units, int L, int dk, int dv) {
     if (umma_supported(dk, dv, L)) return 0;   // one thread block covers a unit
-    if (use_segments(L, dk, dv)) return umma_seg_workspace_bytes(units, L);
+    if (use_segments(units, L, dk, dv)) return umma_seg_workspace_bytes(units, L);
     return umma_long_workspace_bytes(units, L, dk, dv);
 }
 
@@ -41,7 +57,7 @@ cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, cons
                             const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
                             int L, int dk, int dv, void* ws, cudaStream_t stream) {
     if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, 0.f, stream);
-    if (use_segments(L, dk, dv)) return launch_bigla_umma_seg(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
+    if (use_segments(units, L, dk, dv)) return launch_bigla_umma_seg(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
     return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
 }
 
@@ -269,7 +285,8 @@ int vig_last_device_status(void* stream) {
 }
 
 int vig_test_set_kernel_preference(int preference) {
-    if (preference != VIG_TEST_KERNEL_AUTO && preference != VIG_TEST_KERNEL_SIMT && preference != VIG_TEST_KERNEL_CHUNK_TASKS)
+    if (preference != VIG_TEST_KERNEL_AUTO && preference != VIG_TEST_KERNEL_SIMT && preference != VIG_TEST_KERNEL_CHUNK_TASKS &&
+        preference != VIG_TEST_KERNEL_SEGMENTS)
         return VIG_ERR_UNSUPPORTED;
     g_kernel_pref.store(preference, std::memory_order_relaxed);
     return VIG_OK;

@@ -91,16 +91,26 @@ struct UArgs {
     float inv_tau;
 };
 
-// log alpha = logsigmoid(g) / tau (Eq. 5 line 1) for the eight bf16 gate logits of one 16-byte piece, evaluated in
-// fp32 as (min(g, 0) - log(1 + e^{-|g|})) / tau with exp and log from the special-function unit, rounded to bf16.
-__device__ __forceinline__ uint4 log_alpha_piece(uint4 g, float inv_tau) {
-    const float c_log = -0.6931471805599453f * inv_tau;   // log2 -> natural log, over tau, negated
+// log2 alpha = logsigmoid(g) / (tau ln 2) (Eq. 5 line 1, in base 2 so that the operand scaling needs no further
+// multiplication) for the eight bf16 gate logits of one 16-byte piece, evaluated in fp32 as
+// (min(g, 0) log2(e) - log2(1 + e)) / tau with e = e^{-|g|} in (0, 1] from the special-function unit and
+// log2(1 + e) = e p(e), p of degree three (absolute error 1e-4, i.e. 7e-5 / tau in log alpha: below the bf16 rounding
+// that follows), on the FMA pipe: with the logarithm on the special-function unit too, that unit bounds the phase.
+__device__ __forceinline__ float log2_1p_unit(float e) {
+    float p = -0.08476800471544266f;
+    p = fmaf(p, e, 0.3255951702594757f);
+    p = fmaf(p, e, -0.6799444556236267f);
+    p = fmaf(p, e, 1.4390150308609009f);
+    return p * e;
+}
+__device__ __forceinline__ uint4 log2_alpha_piece(uint4 g, float inv_tau) {
+    const float c_lin = kLog2e * inv_tau;
     uint32_t w[4] = {g.x, g.y, g.z, g.w};
 #pragma unroll
     for (int x = 0; x < 4; ++x) {
         const float2 z = unpack_bf16(w[x]);
-        const float l0 = __log2f(1.f + ex2(-fabsf(z.x) * kLog2e)), l1 = __log2f(1.f + ex2(-fabsf(z.y) * kLog2e));
-        w[x] = pack_bf16(fmaf(l0, c_log, fminf(z.x, 0.f) * inv_tau), fmaf(l1, c_log, fminf(z.y, 0.f) * inv_tau));
+        const float l0 = log2_1p_unit(ex2(-fabsf(z.x) * kLog2e)), l1 = log2_1p_unit(ex2(-fabsf(z.y) * kLog2e));
+        w[x] = pack_bf16(fmaf(l0, -inv_tau, fminf(z.x, 0.f) * c_lin), fmaf(l1, -inv_tau, fminf(z.y, 0.f) * c_lin));
     }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
@@ -141,6 +151,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // The warp index goes through a shuffle so that the compiler knows it, and every address and descriptor derived
     // from it, to be uniform across the warp: the operands of tcgen05.mma then stay in uniform registers instead of
     // being moved there one by one before every MMA (measured: -1 us per call).
+    constexpr float kExp = GATES ? 1.f : kLog2e;   // prefix sums of log alpha -> exponent of two
     const int tid = threadIdx.x, lane = tid & 31, warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int c = warp >> 2, wq = warp & 3;            // chunk and row quadrant of this warp
     // Segmented sequences: block b works on segment b % nseg of the units of group b / nseg; the blocks of a group
@@ -285,6 +296,22 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         umma_commit(bar_pfx);
     };
     const int npass_c0 = ks_c0 > 4 ? 2 : 1;
+    // Fused gate preparation (GATES): the two gate tiles of a pair hold the logits g and are rewritten in place as
+    // log2 alpha (the prefix sums, their totals and the range check are then in base 2 as well: kExp = 1), 16-byte pieces dealt out evenly to the threads of the block.  Rows and columns the loads filled with
+    // zeros stay zero (log alpha = 0: no decay, and k = v = 0 there): the forward tile holds token r in row r, the
+    // backward tile token r - 1 (rows 1 .. L).
+    auto prepare_gates = [&](uint32_t pair) {
+        const int per_tile = 4 * min(L + 1, args.rows);   // rows 0 .. L of a tile (as far as it reaches), four pieces each
+#pragma unroll 1
+        for (int x = tid; x < 2 * per_tile; x += kThreads) {
+            const int tile = x >= per_tile, y = x - tile * per_tile, r = y >> 2, pc = y & 3;
+            if ((pc ^ ((r >> 1) & 3)) * 8 >= DK) continue;   // this piece holds padding columns
+            if (tile == 0 ? r >= L : r < 1) continue;
+            uint4* gp = reinterpret_cast<uint4*>(bp + pair + (uint32_t)tile * lay.tile + (uint32_t)r * 64 + pc * 16);
+            *gp = log2_alpha_piece(*gp, args.inv_tau);
+        }
+        fence_async_smem();   // written through the generic proxy, read by the prefix-sum MMAs through the async proxy
+    };
 
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
@@ -309,27 +336,16 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
 
         if constexpr (GATES) {
-            // ---- fused gate preparation: the two gate tiles hold the logits g; thread r rewrites tile row r of both in
-            // place as log alpha.  Rows and columns the loads filled with zeros stay zero (log alpha = 0: no decay, and
-            // k = v = 0 there): the forward tile holds token r in row r, the backward tile token r - 1.
-            wait_bar(bar_g, par);
-            if (tid < args.rows) {
-                const bool f_ok = tid < L, b_ok = tid >= 1 && tid <= L;
-#pragma unroll
-                for (int pc = 0; pc < 4; ++pc) {
-                    if ((pc ^ ((tid >> 1) & 3)) * 8 >= DK) continue;   // this 16-byte piece holds padding columns
-                    uint4* gf = reinterpret_cast<uint4*>(bp + pair_g + (uint32_t)tid * 64 + pc * 16);
-                    uint4* gb = reinterpret_cast<uint4*>(bp + pair_g + lay.tile + (uint32_t)tid * 64 + pc * 16);
-                    if (f_ok) *gf = log_alpha_piece(*gf, args.inv_tau);
-                    if (b_ok) *gb = log_alpha_piece(*gb, args.inv_tau);
-                }
+            // fused gate preparation, unless it was done (and the prefix sums were issued) under the previous unit's epilogue
+            if (!(nc == 2 && *early_gates == (int)it)) {
+                wait_bar(bar_g, par);
+                prepare_gates(pair_g);
+                __syncthreads();
             }
-            fence_async_smem();
-            __syncthreads();
         }
         if (chunk_on) {
             // ---- prefix sums of the log gates (unless they were issued while the previous unit was finishing) ----
-            if (issue_warp && c == 0 && (GATES || !(nc == 2 && *early_gates == (int)it)) && elect_one()) {
+            if (issue_warp && c == 0 && !(nc == 2 && *early_gates == (int)it) && elect_one()) {
                 wait_bar(bar_g, par);
                 issue_prefix(pair_g);
             }
@@ -381,8 +397,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             for (int m = 0; m < 4; ++m) {
                                 // the decaying factors on the special-function unit, the growing ones as their packed reciprocals
                                 const int d0 = 8 * c8 + 2 * m;
-                                const float ex0 = ex2(as_f(pf[hf][d0]) * kLog2e), ex1 = ex2(as_f(pf[hf][d0 + 1]) * kLog2e);
-                                const float ey0 = ex2(as_f(pb[hf][d0]) * kLog2e), ey1 = ex2(as_f(pb[hf][d0 + 1]) * kLog2e);
+                                const float ex0 = ex2(as_f(pf[hf][d0]) * kExp), ex1 = ex2(as_f(pf[hf][d0 + 1]) * kExp);
+                                const float ey0 = ex2(as_f(pb[hf][d0]) * kExp), ey1 = ex2(as_f(pb[hf][d0 + 1]) * kExp);
                                 const uint32_t exp_f = pack_bf16(ex0, ex1), exp_b = pack_bf16(ey0, ey1);
                                 qf[m] = mul_bf16x2(qv[m], exp_f);               // q~> = q e^{b}
                                 kf[m] = mul_bf16x2(kv[m], rcp_bf16x2(exp_f));   // k~> = k e^{-b}
@@ -412,7 +428,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             if (wq == 2) {
                 // range check, one key dim per lane: b and x are smallest at the last row of the chunk
-                const bool out_of_range = dec[(2 * c) * 32 + lane] < -kGateRange || dec[(2 * c + 1) * 32 + lane] < -kGateRange;
+                constexpr float kRange = GATES ? kGateRange * kLog2e : kGateRange;   // the same bound in the base the totals are in
+                const bool out_of_range = dec[(2 * c) * 32 + lane] < -kRange || dec[(2 * c + 1) * 32 + lane] < -kRange;
                 const bool any = __any_sync(0xffffffffu, out_of_range);
                 if (lane == 0) slow_slot[c] = any ? 1 : 0;
             }
@@ -516,7 +533,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state
                     // for chunk 0.  Both are scaled by chunk 0's total decay of their direction, for key dim `lane`.
                     if (warp == 4) named_bar(5, 160);   // chunk 0's threads arrived after writing their totals
-                    const float d = ex2(dec[(warp == 1 ? 0 : 32) + lane] * kLog2e);
+                    const float d = ex2(dec[(warp == 1 ? 0 : 32) + lane] * kExp);
                     uint8_t* st = bp + (warp == 1 ? lay.s_fwd : lay.s_bwd);
 #pragma unroll
                     for (int hb = 0; hb < 2; ++hb) {
@@ -745,7 +762,18 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 umma_commit(bar_mma);
             }
             wait_mma();
-            if (!GATES && warp == 7 && nc == 2 && *early_gates == (int)it + 1 && elect_one()) {
+            if constexpr (GATES) {
+                if (nc == 2) {
+                    // The next unit's gate logits have been on their way since the chunk summaries: every thread prepares
+                    // its share now, so that the prefix sums can be issued under this unit's epilogue as in the un-fused form.
+                    if (*early_gates == (int)it + 1) {
+                        wait_bar(bar_g, par ^ 1);
+                        prepare_gates(pair_qk);
+                    }
+                    if (c == 1 && warp != 7) asm volatile("bar.arrive 6, 256;" ::: "memory");
+                }
+            }
+            if (warp == 7 && nc == 2 && *early_gates == (int)it + 1 && elect_one()) {
                 // The packed scores of both chunks have been consumed (this thread has waited for chunk 1's output batch,
                 // now for chunk 0's): their TMEM columns take the next unit's prefix sums, whose log gates have been on
                 // their way since the chunk summaries.  Warp 7 has the fewest rows to write out.
@@ -754,9 +782,9 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
             if (nc == 2 && warp == 7) {
                 // ... and chunk 0's output has left TMEM block 0, which takes the sums of all four gate blocks
-                named_bar(6, 160);
+                named_bar(6, GATES ? 256 : 160);   // (fused gates: the other warps of chunk 1 have prepared their share too)
                 tc_fence_after();
-                if (!GATES && *early_gates == (int)it + 1 && elect_one()) issue_prefix(pair_qk);   // (fused gates: only once they are prepared)
+                if (*early_gates == (int)it + 1 && elect_one()) issue_prefix(pair_qk);
                 __syncwarp();
             }
             if (ctl_warp && has_next) {
@@ -788,7 +816,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_wait_ld();
                 if (nc == 2 && c == 0) {   // TMEM block 0 is free for the next unit's prefix sums
                     tc_fence_before();
-                    asm volatile("bar.arrive 6, 160;" ::: "memory");
+                    if (GATES) asm volatile("bar.arrive 6, 256;" ::: "memory");
+                    else asm volatile("bar.arrive 6, 160;" ::: "memory");
                 }
                 if (row_live) {
 #pragma unroll

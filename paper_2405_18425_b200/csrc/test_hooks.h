@@ -6,8 +6,10 @@
  *   VIG_TEST_KERNEL_AUTO   the default dispatch
  *   VIG_TEST_KERNEL_SIMT   always the fp32 SIMT recurrence kernel
  *   VIG_TEST_KERNEL_CHUNK_TASKS  sequences of more than 256 tokens always take the three chunk-task launches
- *                          (the default uses them only beyond 32 x 256 tokens).  vig_bigla_workspace_bytes
- *                          follows the setting: query it under the setting the call will run with
+ *   VIG_TEST_KERNEL_SEGMENTS     sequences of 257 .. 8192 tokens always take the segmented single launch
+ *                          (the default chooses between the two by segment count and unit count).
+ *                          vig_bigla_workspace_bytes follows the setting: query it under the setting the call
+ *                          will run with
  * Returns VIG_OK, or VIG_ERR_UNSUPPORTED for an unknown value (the setting is then unchanged). */
 #ifndef VIG_TEST_HOOKS_H
 #define VIG_TEST_HOOKS_H
@@ -16,7 +18,7 @@
 extern "C" {
 #endif
 
-enum vig_test_kernel { VIG_TEST_KERNEL_AUTO = 0, VIG_TEST_KERNEL_SIMT = 2, VIG_TEST_KERNEL_CHUNK_TASKS = 3 };
+enum vig_test_kernel { VIG_TEST_KERNEL_AUTO = 0, VIG_TEST_KERNEL_SIMT = 2, VIG_TEST_KERNEL_CHUNK_TASKS = 3, VIG_TEST_KERNEL_SEGMENTS = 4 };
 int vig_test_set_kernel_preference(int preference);
 
 #ifdef __cplusplus
