@@ -62,13 +62,17 @@ typedef enum vig_dtype { VIG_DTYPE_F32 = 0, VIG_DTYPE_BF16 = 1 } vig_dtype;
  *       dk <= 128, dv <= 256 runs on the fp32 SIMT recurrence kernel (slow, same result
  *       contract).  Tensor-core operands are bf16 with fp32 accumulation; states that cross
  *       a 128-token chunk are rounded to bf16 as tensor-core operands.  A unit whose gates decay
- *       by more than e^-60 inside one chunk of 128 tokens is computed by the exact in-kernel
- *       recurrence instead of the factorised tiles.
+ *       by more than e^-60 inside one chunk of 128 tokens is computed by an in-kernel fp32
+ *       recurrence (Eq. 6 step by step) instead of the factorised tiles.
  * f32:  dk <= 128, dv <= 256; fp32 SIMT recurrence, meant for validation-sized inputs.
- * Sequences of more than 256 tokens are split into 128-token chunks whose boundary states go through
- * scratch memory that the library allocates and frees on `stream` (cudaMallocAsync); use the *_ws
- * form to supply it.  The kernels are launched with programmatic stream serialization: each waits
- * for the work before it in `stream` before it touches global memory.
+ * Sequences of at most 256 tokens run in one launch with a unit per thread block and use no scratch.
+ * Longer ones are cut into 256-token segments (one launch; the blocks of a unit exchange segment
+ * summaries through scratch) or into 128-token chunk tasks (three launches; chunk summaries and
+ * boundary states go through scratch), whichever suits the shape.  The library allocates and frees
+ * that scratch on `stream` from a stream-ordered memory pool of its own (one per device, which keeps
+ * freed memory for later calls instead of returning it to the driver); use the *_ws form to supply it.  The kernels are
+ * launched with programmatic stream serialization: each waits for the work before it in `stream`
+ * before it reads its inputs.
  * Errors: NULL_POINTER, BAD_DIM, UNSUPPORTED, MISALIGNED, CUDA. */
 int vig_bigla_fwd_bf16(const void* q, const void* k, const void* v,
                        const void* log_alpha_fwd, const void* log_alpha_bwd, void* out,
@@ -105,12 +109,14 @@ int vig_bigla_fwd_ws_bf16(const void* q, const void* k, const void* v,
  *     rejected with VIG_ERR_WORKSPACE and nothing is launched; use vig_bigla_fwd_ws_bf16 for it.
  *   - No cudaMalloc, cudaFree or other allocating call is made, by this entry point or beneath it.
  *   - The first call on each device looks up the array's device address (a one-time set-up step for
- *     that device); make that first call with the device current and before starting any stream
+ *     that device, which also makes the runtime load the library's device image, the array included,
+ *     if it has not yet); make that first call with the device current and before starting any stream
  *     capture.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left in it.
- *     The call itself clears the part that must start at zero.  Two calls that overlap on the GPU
- *     (different streams, no ordering between them) race on it and give undefined results: order them.
- * Results are identical to vig_bigla_fwd_bf16.  Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED,
+ *     Nothing in it has to start at zero: every word a call reads to form its result was written
+ *     earlier in the same call.  Two calls that overlap on the GPU (different streams, no ordering
+ *     between them) race on it and give undefined results: order them.
+ * Same kernels and results as vig_bigla_fwd_ws_bf16 with a workspace of that size.  Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED,
  * WORKSPACE, CUDA. */
 #define VIG_STATIC_SCRATCH_BYTES (24u * 1024u * 1024u)
 int vig_bigla_fwd_static_bf16(const void* q, const void* k, const void* v,
@@ -138,7 +144,7 @@ int vig_gate_prep_f32(const void* g_fwd, const void* g_bwd,
  * tile into log alpha in shared memory (fp32 evaluation with exp and log from the special-function unit,
  * rounded to bf16 as the tensor-core operand of the prefix sums: the same rounding point as the un-fused
  * chain).  Longer sequences and other head sizes run gate preparation into scratch the library allocates and
- * frees on `stream`, then the ordinary forward pass.
+ * frees on `stream` (its memory pool), then the ordinary forward pass.
  * Errors: NULL_POINTER, BAD_DIM (also tau), UNSUPPORTED, MISALIGNED, CUDA. */
 int vig_bigla_fwd_gates_bf16(const void* q, const void* k, const void* v,
                              const void* g_fwd, const void* g_bwd, void* out,
@@ -147,9 +153,13 @@ int vig_bigla_fwd_gates_bf16(const void* q, const void* k, const void* v,
 /* ---- Whole path on HOST buffers -------------------------------------------------------------------
  * Gate preparation followed by the BiGLA forward (Eq. 5 line 1 + Eq. 6) for callers whose data
  * lives in host memory.  All seven pointers are HOST pointers (pinned memory makes the copies
- * asynchronous and faster; pageable memory works).  The call copies q, k, v, g_fwd, g_bwd to
- * device memory it allocates on `stream`, runs both kernels there, copies `out` back, frees the
- * device memory and synchronises `stream` before returning, so `out` is valid on return.
+ * asynchronous and faster; pageable memory works).  The call takes device buffers from the library's
+ * memory pool on `stream`, cuts the batch into slices of whole units and runs, on two internal copy
+ * streams ordered with `stream` by events, the copy of one slice to the device, the kernels of the
+ * slice before it (vig_bigla_fwd_gates_bf16, or the two fp32 calls) and the copy of the slice before
+ * that back to `out` at the same time; it returns the device memory to the pool and synchronises
+ * `stream` before returning, so `out` is valid on return.  Results are those of the device entry
+ * points, bit for bit.  Host calls on one device are serialised.
  * `dtype` is a vig_dtype.  Errors: as the device calls, plus CUDA for allocation failures. */
 int vig_bigla_fwd_host(const void* q, const void* k, const void* v,
                        const void* g_fwd, const void* g_bwd, void* out,

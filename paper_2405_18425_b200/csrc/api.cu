@@ -1,6 +1,7 @@
 // C-ABI entry points of libvig_bigla: argument validation, dispatch, host-buffer path, diagnostics.
 #include <atomic>
 #include <cmath>
+#include <mutex>
 
 #include "test_hooks.h"
 #include "vig_internal.h"
@@ -61,6 +62,39 @@ cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, cons
     return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
 }
 
+// ---- scratch the library allocates itself -----------------------------------------------------------------------
+// Stream-ordered allocations come from a memory pool of the library's own, one per device, whose release threshold
+// keeps freed memory for the next call: with the default pool's threshold of zero every synchronisation hands the
+// memory back to the driver and the next call maps it afresh (tens of microseconds per call, milliseconds for the
+// buffers of the host path).  The application's default pool keeps whatever settings it was given.
+static cudaMemPool_t device_pool() {
+    static cudaMemPool_t pools[64] = {};
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!pools[dev]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t pool = nullptr;
+        unsigned long long keep = ~0ull;
+        if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) return nullptr;
+        if (cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep) != cudaSuccess) {
+            cudaMemPoolDestroy(pool);
+            return nullptr;
+        }
+        pools[dev] = pool;
+    }
+    return pools[dev];
+}
+static cudaError_t pool_alloc(void** p, size_t bytes, cudaStream_t stream) {
+    cudaMemPool_t pool = device_pool();
+    return pool ? cudaMallocFromPoolAsync(p, bytes, pool, stream) : cudaErrorMemoryAllocation;
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Shared checks of the forward entry points.  Returns VIG_OK with *empty = true for B*H*L == 0.
@@ -93,7 +127,7 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
         if (empty) return VIG_OK;
         void* scratch = ws;
         if (own_ws && need > 0) {
-            if (cudaMallocAsync(&scratch, need, stream) != cudaSuccess) return VIG_ERR_CUDA;
+            if (pool_alloc(&scratch, need, stream) != cudaSuccess) return VIG_ERR_CUDA;
         }
         cudaError_t e = launch_bigla_tc(q_, k_, v_, f_, b_, (bf*)out, units, L, dk, dv, scratch, stream);
         if (own_ws && need > 0) {
@@ -128,7 +162,7 @@ static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, cons
     const size_t n = (size_t)units * L * dk;
     const size_t gate_bytes = (n * sizeof(bf) + 255) / 256 * 256;
     char* la = nullptr;
-    if (cudaMallocAsync((void**)&la, 2 * gate_bytes, stream) != cudaSuccess) return VIG_ERR_CUDA;
+    if (pool_alloc((void**)&la, 2 * gate_bytes, stream) != cudaSuccess) return VIG_ERR_CUDA;
     st = vig_gate_prep_bf16(g_f, g_b, la, la + gate_bytes, B, H, L, dk, tau, stream);
     if (st == VIG_OK) st = vig_bigla_fwd_bf16(q, k, v, la, la + gate_bytes, out, B, H, L, dk, dv, stream);
     if (cudaFreeAsync(la, stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
@@ -166,6 +200,36 @@ static int gate_prep_impl(const void* g_f, const void* g_b, void* la_f, void* la
     const long long n = (long long)B * H * L * dk;
     cudaError_t e = launch_gate_prep<T>((const T*)g_f, (const T*)g_b, (T*)la_f, (T*)la_b, n, tau, stream);
     return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
+// ---- host-buffer path: per device, two copy streams and the events that order them with the caller's stream -------
+constexpr int kHostSlices = 4;
+struct HostPath {
+    std::mutex mu;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_done_in = nullptr, ev_done_out = nullptr, ev_in[kHostSlices] = {}, ev_k[kHostSlices] = {};
+    bool ready = false;
+};
+static HostPath* host_path() {
+    static HostPath per_device[64];
+    static std::mutex init_mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPath* hp = &per_device[dev];
+    std::lock_guard<std::mutex> lock(init_mu);
+    if (!hp->ready) {
+        bool ok = cudaStreamCreateWithFlags(&hp->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&hp->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp->ev_done_in, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&hp->ev_done_out, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kHostSlices; ++i)
+            ok = cudaEventCreateWithFlags(&hp->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp->ev_k[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        hp->ready = true;
+    }
+    return hp;
 }
 
 }  // namespace vig
@@ -227,32 +291,55 @@ int vig_bigla_fwd_host(const void* q, const void* k, const void* v, const void* 
     if (dtype != VIG_DTYPE_F32 && dtype != VIG_DTYPE_BF16) return VIG_ERR_UNSUPPORTED;
     if (dtype == VIG_DTYPE_F32 ? !recurrence_supported(dk, dv) : !(tc_supported(dk, dv) || recurrence_supported(dk, dv)))
         return VIG_ERR_UNSUPPORTED;
+    if ((long long)B * H > 0x7fffffffLL) return VIG_ERR_UNSUPPORTED;
     if (B == 0 || H == 0 || L == 0) return VIG_OK;
+    HostPath* hp = host_path();
+    if (!hp) return VIG_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(hp->mu);   // the streams and events of the device serve one host call at a time
     const size_t es = dtype == VIG_DTYPE_F32 ? 4 : 2;
-    const size_t tok = (size_t)B * H * L;
+    const long long units = (long long)B * H;
+    const size_t unit_k = (size_t)L * dk * es, unit_v = (size_t)L * dv * es;
     // every slab is rounded up to 256 bytes so that all device pointers stay aligned
-    const size_t nk = (tok * dk * es + 255) / 256 * 256, nv = (tok * dv * es + 255) / 256 * 256;
+    const size_t nk = (units * unit_k + 255) / 256 * 256, nv = (units * unit_v + 255) / 256 * 256;
     char* base = nullptr;
-    if (cudaMallocAsync((void**)&base, 4 * nk + 2 * nv, stream) != cudaSuccess) return VIG_ERR_CUDA;
+    if (pool_alloc((void**)&base, 4 * nk + 2 * nv, stream) != cudaSuccess) return VIG_ERR_CUDA;
     char *dq = base, *dk_ = base + nk, *dgf = base + 2 * nk, *dgb = base + 3 * nk, *dv_ = base + 4 * nk,
          *dout = base + 4 * nk + nv;
+    // Slices of whole units: the copy of slice i + 1 to the device, the kernels of slice i and the copy of slice i - 1
+    // back run at the same time (the host link carries both directions at once).  A slice offset must keep the 16-byte
+    // alignment of the device pointers: unit sizes are multiples of 16 bytes whenever dk and dv are multiples of
+    // 8 (bf16) or 4 (fp32); otherwise the call runs as one slice.
+    int nsl = (unit_k % 16 == 0 && unit_v % 16 == 0 && units * (4 * unit_k + 2 * unit_v) >= (4u << 20)) ? kHostSlices : 1;
+    if (nsl > units) nsl = (int)units;
     int st = VIG_OK;
-    bool ok = cudaMemcpyAsync(dq, q, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-              cudaMemcpyAsync(dk_, k, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-              cudaMemcpyAsync(dv_, v, tok * dv * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-              cudaMemcpyAsync(dgf, g_fwd, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-              cudaMemcpyAsync(dgb, g_bwd, tok * dk * es, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    if (!ok) st = VIG_ERR_CUDA;
-    if (st == VIG_OK) {
-        st = dtype == VIG_DTYPE_F32 ? vig_gate_prep_f32(dgf, dgb, dgf, dgb, B, H, L, dk, tau, stream_)
-                                    : vig_gate_prep_bf16(dgf, dgb, dgf, dgb, B, H, L, dk, tau, stream_);
+    bool ok = cudaEventRecord(hp->ev_start, stream) == cudaSuccess &&
+              cudaStreamWaitEvent(hp->s_in, hp->ev_start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(hp->s_out, hp->ev_start, 0) == cudaSuccess;
+    for (int i = 0; ok && i < nsl && st == VIG_OK; ++i) {
+        const long long u0 = units * i / nsl, u1 = units * (i + 1) / nsl, nu = u1 - u0;
+        const size_t ok_ = (size_t)u0 * unit_k, ov = (size_t)u0 * unit_v;
+        ok = cudaMemcpyAsync(dgf + ok_, (const char*)g_fwd + ok_, nu * unit_k, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess &&
+             cudaMemcpyAsync(dgb + ok_, (const char*)g_bwd + ok_, nu * unit_k, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess &&
+             cudaMemcpyAsync(dq + ok_, (const char*)q + ok_, nu * unit_k, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess &&
+             cudaMemcpyAsync(dk_ + ok_, (const char*)k + ok_, nu * unit_k, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess &&
+             cudaMemcpyAsync(dv_ + ov, (const char*)v + ov, nu * unit_v, cudaMemcpyHostToDevice, hp->s_in) == cudaSuccess &&
+             cudaEventRecord(hp->ev_in[i], hp->s_in) == cudaSuccess && cudaStreamWaitEvent(stream, hp->ev_in[i], 0) == cudaSuccess;
+        if (!ok) break;
+        if (dtype == VIG_DTYPE_F32) {
+            st = vig_gate_prep_f32(dgf + ok_, dgb + ok_, dgf + ok_, dgb + ok_, (int)nu, 1, L, dk, tau, stream_);
+            if (st == VIG_OK) st = vig_bigla_fwd_f32(dq + ok_, dk_ + ok_, dv_ + ov, dgf + ok_, dgb + ok_, dout + ov, (int)nu, 1, L, dk, dv, stream_);
+        } else {
+            st = vig_bigla_fwd_gates_bf16(dq + ok_, dk_ + ok_, dv_ + ov, dgf + ok_, dgb + ok_, dout + ov, (int)nu, 1, L, dk, dv, tau, stream_);
+        }
+        if (st != VIG_OK) break;
+        ok = cudaEventRecord(hp->ev_k[i], stream) == cudaSuccess && cudaStreamWaitEvent(hp->s_out, hp->ev_k[i], 0) == cudaSuccess &&
+             cudaMemcpyAsync((char*)out + ov, dout + ov, nu * unit_v, cudaMemcpyDeviceToHost, hp->s_out) == cudaSuccess;
     }
-    if (st == VIG_OK) {
-        st = dtype == VIG_DTYPE_F32 ? vig_bigla_fwd_f32(dq, dk_, dv_, dgf, dgb, dout, B, H, L, dk, dv, stream_)
-                                    : vig_bigla_fwd_bf16(dq, dk_, dv_, dgf, dgb, dout, B, H, L, dk, dv, stream_);
-    }
-    if (st == VIG_OK && cudaMemcpyAsync(out, dout, tok * dv * es, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-        st = VIG_ERR_CUDA;
+    // the caller's stream takes over again once both copy streams have drained (also after an error, so that the
+    // buffer is not freed under a copy in flight)
+    ok = (cudaEventRecord(hp->ev_done_in, hp->s_in) == cudaSuccess) & (cudaEventRecord(hp->ev_done_out, hp->s_out) == cudaSuccess) &
+         (cudaStreamWaitEvent(stream, hp->ev_done_in, 0) == cudaSuccess) & (cudaStreamWaitEvent(stream, hp->ev_done_out, 0) == cudaSuccess) & ok;
+    if (!ok && st == VIG_OK) st = VIG_ERR_CUDA;
     if (cudaFreeAsync(base, stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
     return st;

@@ -11,7 +11,7 @@
 //      S<_in(m) = d<(m) R(m + 1) (q~< = q e^{-x} lacks the chunk's own decay), in fp32; every incoming state is
 //      written out as the bf16 shared-memory image the next launch copies in with one bulk copy;
 //   3. main: per chunk, out = ( P v + q~> S>_in + q~< S<_in ) / 2 with P = tril(q~> k~>^T) + triu(q~< k~<^T).
-// Blocks are persistent (three per SM, 128 threads, 128 TMEM columns each) and walk over the tasks; thread r
+// Blocks are persistent (four per SM, 128 threads, 128 TMEM columns each) and walk over the tasks; thread r
 // owns token r of the chunk in every element-wise phase.  All products are tcgen05.mma with M = 128.
 #include <cuda.h>
 

@@ -1,4 +1,6 @@
 // Gate preparation: log alpha = logsigmoid(g) / tau (paper Eq. 5 line 1), both directions in one launch.
+#include <atomic>
+
 #include "ptx.cuh"
 #include "vig_internal.h"
 
@@ -77,7 +79,17 @@ cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long 
     const int threads = 256;
     long long blocks = (n / V + threads - 1) / threads;
     if (blocks < 1) blocks = 1;
-    if (blocks > 148 * 4) blocks = 148 * 4;   // both directions together: eight blocks per SM
+    // both directions together: eight blocks per SM (the SM count of the current device, queried once per device)
+    static std::atomic<int> sms_of[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    int sms = sms_of[dev].load(std::memory_order_relaxed);
+    if (sms == 0) {
+        const cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        sms_of[dev].store(sms, std::memory_order_relaxed);
+    }
+    if (blocks > 4LL * sms) blocks = 4LL * sms;
     const cudaError_t le = launch_pdl(gate_prep_kernel<T>, dim3((unsigned)blocks, 2), dim3(threads), 0, stream, g_f, g_b, la_f, la_b, n, 1.0f / tau);
     count_launch();
     return le != cudaSuccess ? le : cudaGetLastError();

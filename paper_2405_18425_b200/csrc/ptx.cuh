@@ -1,4 +1,4 @@
-// Inline-PTX wrappers shared by the tensor-core kernels (mbarrier, TMA, ldmatrix, mma.sync, packing)
+// Inline-PTX wrappers shared by the kernels (mbarrier, TMA, packing, programmatic dependent launch)
 // and the address function of TMA-swizzled shared-memory tiles.
 #pragma once
 #include <cuda.h>
@@ -54,23 +54,6 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int 
                  "r"(x), "r"(y), "r"(z), "r"(src)
                  : "memory");
 }
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -86,19 +69,11 @@ __device__ __forceinline__ float2 unpack_bf16(uint32_t u) {
 __device__ __forceinline__ void named_bar(int id, int count) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
 }
-__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
-    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-
 // Programmatic dependent launch.  `pdl_launch_dependents`: the next kernel in the stream, if it was launched with
 // programmatic stream serialization, may start its prologue once every block of this grid has executed this (or
 // exited).  `pdl_wait`: blocks until every kernel this grid depends on has completed and its memory operations are
-// visible; a no-op for an ordinary launch.  The kernels here execute it before their first global-memory access.
+// visible; a no-op for an ordinary launch.  The kernels here execute it before their first global-memory read into
+// shared memory or registers and before any write; prefetches into L2, which consume nothing, may precede it.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <stdint.h>
 
 namespace vig {
 
@@ -22,7 +23,7 @@ inline EncodeFn encode_fn() {
 }
 
 // [units][L][d] bf16 tensor, box = [1][rows][row_elems] with row_elems*2 bytes = the swizzle span.
-inline bool make_map(CUtensorMap* map, const void* ptr, long long units, int L, int d, int row_elems, int rows) {
+inline bool encode_map(CUtensorMap* map, const void* ptr, long long units, int L, int d, int row_elems, int rows) {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)L, (cuuint64_t)units};
@@ -35,6 +36,31 @@ inline bool make_map(CUtensorMap* map, const void* ptr, long long units, int L, 
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The same, through a small cache per host thread: a tensor map is a pure function of the six arguments (it holds the
+// address and the shape, nothing of the device's state), and a caller that runs the same buffers again and again - a
+// serving loop, a benchmark - would otherwise pay six driver calls of a microsecond or two per forward call.
+inline bool make_map(CUtensorMap* map, const void* ptr, long long units, int L, int d, int row_elems, int rows) {
+    struct Entry {
+        const void* ptr;
+        long long units;
+        int L, d, row_elems, rows;
+        bool valid;
+        CUtensorMap map;
+    };
+    constexpr int kEntries = 64;   // direct-mapped by a hash of the address: six maps per call, ten buffer sets and more fit
+    thread_local Entry cache[kEntries] = {};
+    const uintptr_t a = reinterpret_cast<uintptr_t>(ptr);
+    Entry& e = cache[((a >> 8) ^ (a >> 17) ^ (uintptr_t)(rows * 7 + row_elems)) % kEntries];
+    if (e.valid && e.ptr == ptr && e.units == units && e.L == L && e.d == d && e.row_elems == row_elems && e.rows == rows) {
+        *map = e.map;
+        return true;
+    }
+    if (!encode_map(map, ptr, units, L, d, row_elems, rows)) return false;
+    e.ptr = ptr; e.units = units; e.L = L; e.d = d; e.row_elems = row_elems; e.rows = rows; e.valid = true;
+    e.map = *map;
+    return true;
 }
 
 }  // namespace vig

@@ -34,18 +34,24 @@ def test_static_scratch_entry_matches_regular_entry_twice():
     args_a = _problem(11, 5, 1500, 24, 48)      # 12 segments per unit: needs the scratch
     args_b = _problem(12, 3, 777, 32, 64)       # a different shape right after, same shared scratch
     assert 0 < vig.vig_bigla_workspace_bytes(5, 1, 1500, 24, 48) <= STATIC_BYTES
-    for args in (args_a, args_b, args_a):
+    outs = {id(a): torch.full_like(a[2], float("nan")) for a in (args_a, args_b)}   # made before the free-memory readings
+    for n, args in enumerate((args_a, args_b, args_a)):
         q, k, v, la_f, la_b = args
         ref = torch.full_like(v, float("nan"))
         vig.vig_bigla_fwd_bf16(q, k, v, la_f, la_b, ref)
         B, H, L, dk = q.shape
-        for _ in range(2):                       # two calls in a row reuse whatever the last one left behind
-            out = torch.full_like(v, float("nan"))
+        for rep in range(2):                     # two calls in a row reuse whatever the last one left behind
+            out = outs[id(args)]
+            out.fill_(float("nan"))
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             st = lib.vig_bigla_fwd_static_bf16(q.data_ptr(), k.data_ptr(), v.data_ptr(), la_f.data_ptr(),
                                                la_b.data_ptr(), out.data_ptr(), B, H, L, dk, v.shape[3],
                                                torch.cuda.current_stream().cuda_stream)
             assert st == 0
             torch.cuda.synchronize()
+            if n > 0 or rep > 0:                 # past the first call (one-time set-up): the device's free memory does not move
+                assert torch.cuda.mem_get_info()[0] == free_before
             got, want = out.float().cpu().numpy(), ref.float().cpu().numpy()
             assert np.isfinite(got).all()
             assert np.abs(got - want).max() <= 2e-2 * np.abs(want).max()
