@@ -25,6 +25,8 @@ from .binding import (  # noqa: F401
     vig_kernel_launch_count,
     vig_last_device_status,
     vig_test_set_kernel_preference,
+    vig_test_take_fallback_count,
+    vig_test_expire_next_wait,
     VIG_TEST_KERNEL_AUTO,
     VIG_TEST_KERNEL_SIMT,
     VIG_TEST_KERNEL_CHUNK_TASKS,

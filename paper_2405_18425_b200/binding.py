@@ -59,6 +59,10 @@ def load() -> ctypes.CDLL:
         lib.vig_last_device_status.restype = ci
         lib.vig_test_set_kernel_preference.argtypes = [ci]
         lib.vig_test_set_kernel_preference.restype = ci
+        lib.vig_test_take_fallback_count.argtypes = [vp]
+        lib.vig_test_take_fallback_count.restype = ci
+        lib.vig_test_expire_next_wait.argtypes = []
+        lib.vig_test_expire_next_wait.restype = None
         lib.vig_kernel_launch_count.argtypes = []
         lib.vig_kernel_launch_count.restype = ctypes.c_ulonglong
         _lib = lib
@@ -193,6 +197,16 @@ VIG_TEST_KERNEL_AUTO, VIG_TEST_KERNEL_SIMT, VIG_TEST_KERNEL_CHUNK_TASKS, VIG_TES
 def vig_test_set_kernel_preference(preference: int) -> None:
     """Test hook (csrc/test_hooks.h; not part of the public C ABI): forces a kernel family process-wide."""
     _check(load().vig_test_set_kernel_preference(int(preference)), "vig_test_set_kernel_preference")
+
+
+def vig_test_take_fallback_count(stream=None) -> int:
+    """Test hook: units handed to the in-kernel recurrence since the last reading (reads and clears)."""
+    return int(load().vig_test_take_fallback_count(_stream(stream)))
+
+
+def vig_test_expire_next_wait() -> None:
+    """Test hook: the next single-block tensor-core launch lets one bounded device-side wait run out."""
+    load().vig_test_expire_next_wait()
 
 
 def vig_kernel_launch_count() -> int:

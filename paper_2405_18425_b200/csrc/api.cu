@@ -8,7 +8,11 @@
 
 namespace vig {
 
-__device__ int g_device_status = 0;
+// [0]: the device status word (bit flags, kDevStatus*);  [1]: units the tensor-core kernels handed to their in-kernel
+// recurrence since the counter was last read (a test aid: kernels find it one word behind the status word).
+__device__ int g_device_status[2] = {0, 0};
+static std::atomic<int> g_expire_next_wait{0};   // test hook: the next single-block launch lets one bounded wait run out
+int take_expire_next_wait() { return g_expire_next_wait.exchange(0, std::memory_order_relaxed); }
 
 static std::atomic<unsigned long long> g_launches{0};
 static std::atomic<int> g_kernel_pref{VIG_TEST_KERNEL_AUTO};   // changed by the test hook only
@@ -362,10 +366,10 @@ const char* vig_status_string(int status) {
 int vig_last_device_status(void* stream) {
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return VIG_ERR_CUDA;
     int word = 0;
-    if (cudaMemcpyFromSymbol(&word, g_device_status, sizeof(int)) != cudaSuccess) return VIG_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&word, g_device_status, sizeof(int), 0) != cudaSuccess) return VIG_ERR_CUDA;
     if (word != 0) {
         const int zero = 0;
-        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return VIG_ERR_CUDA;
+        if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int), 0) != cudaSuccess) return VIG_ERR_CUDA;
     }
     if (word & kDevStatusInternal) return VIG_ERR_CUDA;
     return (word & kDevStatusTimeout) ? VIG_ERR_DEVICE_TIMEOUT : VIG_OK;
@@ -378,6 +382,18 @@ int vig_test_set_kernel_preference(int preference) {
     g_kernel_pref.store(preference, std::memory_order_relaxed);
     return VIG_OK;
 }
+
+int vig_test_take_fallback_count(void* stream) {
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return VIG_ERR_CUDA;
+    int n = 0;
+    const int zero = 0;
+    if (cudaMemcpyFromSymbol(&n, g_device_status, sizeof(int), sizeof(int)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int), sizeof(int)) != cudaSuccess)
+        return VIG_ERR_CUDA;
+    return n;
+}
+
+void vig_test_expire_next_wait(void) { g_expire_next_wait.store(1, std::memory_order_relaxed); }
 
 unsigned long long vig_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -89,6 +89,7 @@ struct UArgs {
     unsigned long long nonce;     // marks the flags of this call
     // fused gate preparation only (GATES): la_f / la_b hold the gate logits g, and log alpha = logsigmoid(g) / tau
     float inv_tau;
+    int expire_wait;   // test hook: every block lets one bounded wait, on an mbarrier nothing completes, run out
 };
 
 // log2 alpha = logsigmoid(g) / (tau ln 2) (Eq. 5 line 1, in base 2 so that the operand scaling needs no further
@@ -222,6 +223,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
         mbar_init(bar_pfx, 1);
+        mbar_init(bar_g + 80, 1);   // never completed: only the test hook waits on it
         *time_flag = 0;
         *early_gates = -1;
         *unit_slow_slot = 0;
@@ -264,8 +266,8 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // A bounded wait that expires raises the flag and lets the block finish the unit on whatever it has:
     // every later wait is bounded too, nothing more is stored, and the host sees the device status word.
-    auto wait_bar = [&](uint32_t bar, uint32_t parity) {
-        if (!mbar_wait_bounded(bar, parity)) *time_flag = 1;
+    auto wait_bar = [&](uint32_t bar, uint32_t parity, uint32_t limit = 1u << 21) {
+        if (!mbar_wait_bounded(bar, parity, limit)) *time_flag = 1;
     };
     auto wait_mma = [&]() {
         wait_bar(bar_mma, mma_phase & 1);
@@ -313,6 +315,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         fence_async_smem();   // written through the generic proxy, read by the prefix-sum MMAs through the async proxy
     };
 
+    if (args.expire_wait && tid == 0) wait_bar(bar_g + 80, 0, 64);   // test hook: this wait cannot succeed
     // ---- the block walks over its units; the loads of the next one are issued while this one is stored ----
     uint32_t it = 0;
     bool v_load_pending = false;      // control warp (uniform in it): the v tile of the current unit has not been requested yet
@@ -863,6 +866,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             // (its scratch overlays the tiles, so the next loads wait until it is done).
             // (segmented sequences: the block of the first segment redoes the whole unit, the others store nothing)
             if (seg == 0) {
+                if (tid == 0) atomicAdd(args.dev_status + 1, 1);   // units handed to the recurrence (read by the tests)
                 const size_t ok = (size_t)unit * args.L * DK, ov = (size_t)unit * args.L * DV;
                 recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
                                                args.out + ov, args.L, DK, DV, reinterpret_cast<float*>(bp), GATES ? args.inv_tau : 0.f);
@@ -936,6 +940,7 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows; a.units = units;
     a.nseg = 1;
     a.inv_tau = GATES ? 1.f / tau : 0.f;
+    a.expire_wait = take_expire_next_wait();
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
     // The MMAs of chunk 1 read 128 rows of the operand tiles from row 128 on, i.e. up to (256 - rows) * 64

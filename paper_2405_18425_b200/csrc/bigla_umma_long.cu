@@ -494,6 +494,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             // the first chunk's task redoes the whole unit by the recurrence (its scratch overlays the tiles, so the
             // next loads wait until it is done); the other chunks of the unit store nothing
             if (m == 0) {
+                if (tid == 0) atomicAdd(args.dev_status + 1, 1);   // units handed to the recurrence (read by the tests)
                 const size_t ok = (size_t)unit * L * DK, ov = (size_t)unit * L * DV;
                 recurrence_unit<__nv_bfloat16>(args.q + ok, args.k + ok, args.v + ov, args.la_f + ok, args.la_b + ok,
                                                args.out + ov, L, DK, DV, reinterpret_cast<float*>(bp));

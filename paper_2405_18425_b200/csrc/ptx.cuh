@@ -31,9 +31,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait: polls without backing off for the first few microseconds (the common case: an MMA
 // batch or a TMA load in flight), then sleeps between polls; gives up after about a quarter of a
 // second and reports it.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = 1u << 21) {
 #pragma unroll 1   // many call sites: an unrolled poll loop would multiply the kernels' code size
-    for (uint32_t spin = 0; spin < (1u << 21); ++spin) {
+    for (uint32_t spin = 0; spin < limit; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
         if (spin > 4096) __nanosleep(128);
     }

@@ -21,6 +21,17 @@ extern "C" {
 enum vig_test_kernel { VIG_TEST_KERNEL_AUTO = 0, VIG_TEST_KERNEL_SIMT = 2, VIG_TEST_KERNEL_CHUNK_TASKS = 3, VIG_TEST_KERNEL_SEGMENTS = 4 };
 int vig_test_set_kernel_preference(int preference);
 
+/* Synchronises `stream`, then returns and clears the number of (batch, head) units that the tensor-core kernels of the
+ * current device handed to their in-kernel fp32 recurrence because a gate left the range of the factorised tiles
+ * (negative: a vig_status error). */
+int vig_test_take_fallback_count(void* stream);
+
+/* The next launch of the single-block tensor-core kernel (sequences of at most 256 tokens) makes every block wait, with
+ * a limit of a few dozen polls, on an mbarrier that nothing ever completes: the bounded wait runs out within
+ * microseconds, the blocks finish their unit without storing anything, and vig_last_device_status reports
+ * VIG_ERR_DEVICE_TIMEOUT.  Nothing faults and nothing spins beyond that limit. */
+void vig_test_expire_next_wait(void);
+
 #ifdef __cplusplus
 }
 #endif

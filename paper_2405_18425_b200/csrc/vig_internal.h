@@ -12,7 +12,9 @@ namespace vig {
 // Device status word: bit flags set by kernels whose bounded waits expire.
 constexpr int kDevStatusTimeout = 1;
 constexpr int kDevStatusInternal = 2;   // a kernel found its own set-up inconsistent (reported as VIG_ERR_CUDA)
-int* device_status_ptr();            // device address of the status word of the current device (NULL on error)
+int* device_status_ptr();            // device address of the status word of the current device (NULL on error);
+                                     // one int behind it: the count of units handed to the in-kernel recurrence
+int take_expire_next_wait();         // test hook: 1 once after vig_test_expire_next_wait(), else 0
 void count_launch(unsigned n = 1);   // bumps the process-wide launch counter
 
 // ---- fp32 SIMT recurrence (Eq. 6 evaluated step by step), any dk <= 128, dv <= 256 ----

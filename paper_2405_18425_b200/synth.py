@@ -66,7 +66,24 @@ CONFIGS = (
     BiglaConfig("vig_b_224", B=64, H=12, L=196, dk=32, dv=64, dtype="bf16", gate_mean=2.0, seed=3),
     BiglaConfig("vig_t_1024", B=8, H=4, L=4096, dk=24, dv=48, dtype="bf16", gate_mean=0.0, seed=4),
 )
-CONFIG_BY_NAME = {c.name: c for c in CONFIGS}
+
+# Second workload: the resolution sweep of the paper's efficiency figure (224^2 .. 2048^2 at patch size 16:
+# L = 196 .. 16384, ViG-T-like heads, batch shrunk as the image grows so that the token count stays near 32 K)
+# and the four stages of the hierarchical ViG-H-T at 224^2 (patch size 4: L = 3136, 784, 196, 49; channels
+# 96 .. 768 over 3 .. 24 heads, i.e. dk = 16, dv = 32 per head).  Same value distributions as the benchmark
+# configurations; they stand in for activations of those model variants, which are not available.
+SWEEP_CONFIGS = (
+    BiglaConfig("res_224", B=168, H=4, L=196, dk=24, dv=48, dtype="bf16", gate_mean=0.0, seed=11),
+    BiglaConfig("res_448", B=42, H=4, L=784, dk=24, dv=48, dtype="bf16", gate_mean=0.0, seed=12),
+    BiglaConfig("res_896", B=10, H=4, L=3136, dk=24, dv=48, dtype="bf16", gate_mean=0.0, seed=13),
+    BiglaConfig("res_1024", B=8, H=4, L=4096, dk=24, dv=48, dtype="bf16", gate_mean=0.0, seed=14),
+    BiglaConfig("res_2048", B=2, H=4, L=16384, dk=24, dv=48, dtype="bf16", gate_mean=0.0, seed=15),
+    BiglaConfig("vig_h_t_stage1", B=16, H=3, L=3136, dk=16, dv=32, dtype="bf16", gate_mean=0.0, seed=21),
+    BiglaConfig("vig_h_t_stage2", B=16, H=6, L=784, dk=16, dv=32, dtype="bf16", gate_mean=0.0, seed=22),
+    BiglaConfig("vig_h_t_stage3", B=16, H=12, L=196, dk=16, dv=32, dtype="bf16", gate_mean=0.0, seed=23),
+    BiglaConfig("vig_h_t_stage4", B=16, H=24, L=49, dk=16, dv=32, dtype="bf16", gate_mean=0.0, seed=24),
+)
+CONFIG_BY_NAME = {c.name: c for c in CONFIGS + SWEEP_CONFIGS}
 
 
 def _splitmix64(x: np.ndarray) -> np.ndarray:
