@@ -61,6 +61,7 @@ struct ULayout {
     uint32_t s_bwd;    // bf16 state entering chunk 0 from the right  (segmented sequences keep their states elsewhere)
     uint32_t zf;       // 0/1 tile of the prefix sums
     uint32_t dec;      // [2 chunks][2][32] fp32 totals of the log gates: b and x at the chunk's last row
+    uint32_t masks;    // 0 / 1 masks of the diagonal score block (kMaskBytes)
     uint32_t misc;     // six mbarriers, TMEM slot, flags
     uint32_t total;
 };
@@ -72,7 +73,8 @@ __host__ __device__ inline ULayout make_layout(int rows, bool seg) {
     l.s_bwd = l.s_fwd + (seg ? 0 : 32 * 128);
     l.zf = l.s_bwd + (seg ? 0 : 32 * 128);
     l.dec = l.zf + kZBytes;
-    l.misc = l.dec + 4 * 32 * 4;
+    l.masks = l.dec + 4 * 32 * 4;
+    l.misc = l.masks + kMaskBytes;
     l.total = l.misc + 128;
     return l;
 }
@@ -237,6 +239,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
     }
     build_zero_one_tile(bp + lay.zf, tid);
+    build_diag_masks(bp + lay.masks, tid);
     // Tile rows the loads never reach (from `rows` up to the 256-row pitch) are K rows of the prefix-sum product
     // of chunk 1: they must be finite, and nothing but the recurrence scratch ever writes them again.
     auto zero_tail_rows = [&]() {
@@ -466,7 +469,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 wait_mma();
                 if (warp_live) {
                     uint32_t pk[16];
-                    combine_any(2 * p, wq, true, rc, rc + 64, lane, pk);
+                    combine_any(2 * p, wq, true, rc, rc + 64, lane, base + lay.masks, pk);
                     if (p == 0) {
 #pragma unroll
                         for (int e = 0; e < 16; ++e) hold[e] = pk[e];
@@ -480,7 +483,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 16; ++e) hold[e] = pk[e];
                     }
-                    combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, pk);
+                    combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, base + lay.masks, pk);
                     if (p == 0) {
 #pragma unroll
                         for (int e = 0; e < 16; ++e) hold[16 + e] = pk[e];

@@ -388,7 +388,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (p == 0 && ctl_warp && elect_one()) load_states(task);   // rows 0..63 of k~> and k~< have been read for the last time
             if (warp_live) {
                 uint32_t pk[16];
-                combine_any(2 * p, wq, true, rc, rc + 64, lane, pk);
+                combine_any(2 * p, wq, true, rc, rc + 64, lane, 0u, pk);   // (no room for the mask table at four blocks per SM: selects)
                 if (p == 0) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) hold[e] = pk[e];
@@ -402,7 +402,7 @@ bigla_long_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
                     for (int e = 0; e < 16; ++e) hold[e] = pk[e];
                 }
-                combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, pk);
+                combine_any(2 * p + 1, wq, 64 * p + 32 < nkeys, rc + 32, rc + 96, lane, 0u, pk);   // (no room for the mask table at four blocks per SM: selects)
                 if (p == 0) {
 #pragma unroll
                     for (int e = 0; e < 16; ++e) hold[16 + e] = pk[e];

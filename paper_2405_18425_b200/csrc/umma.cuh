@@ -81,18 +81,41 @@ __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
 }
 __device__ __forceinline__ float as_f(uint32_t u) { return __uint_as_float(u); }
 
+// Masks of the diagonal 32 x 32 block of P, as packed bf16 pairs of 0 and 1.  For the row of lane t and the column
+// pair (2e, 2e + 1) only d = t - 2e matters: the forward scores count for columns <= t (low half if d >= 0, high half if
+// d >= 1), the backward scores for columns >= t (low half if d <= 0, high half if d <= 1).  The table holds, per parity
+// of t, the 31 possible pairs (forward mask, backward mask) at index e - (t >> 1) + 15, so that a lane steps through
+// consecutive entries as e grows.  kMaskBytes of shared memory; threads 0..61 of the block write it.
+constexpr uint32_t kMaskBytes = 512;
+__device__ __forceinline__ void build_diag_masks(uint8_t* tab, int tid) {
+    if (tid < 62) {
+        const int par = tid / 31, n = tid - par * 31, d = 2 * (15 - n) + par;
+        const uint32_t fw = (d >= 0 ? 0x3F80u : 0u) | (d >= 1 ? 0x3F800000u : 0u);
+        const uint32_t bw = (d <= 0 ? 0x3F80u : 0u) | (d <= 1 ? 0x3F800000u : 0u);
+        *reinterpret_cast<uint2*>(tab + (par * 31 + n) * 8) = make_uint2(fw, bw);
+    }
+}
+__device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // Packed bf16 values of one 32-column block of P for this thread's row.  REL < 0: the block lies left
 // of the diagonal block (forward scores only), REL > 0: right of it (backward only), REL == 0: the
-// diagonal block, forward part masked to s <= t, backward part to s >= t, summed in fp32.
+// diagonal block: forward scores for s <= t plus backward scores for s >= t, taken as packed products with the 0 / 1
+// masks above (exact off the diagonal; on it the two bf16 values are added and rounded once more).  The scores outside
+// the masks are finite: the range check of the gates bounds the growing factors.
 template <int REL>
-__device__ __forceinline__ void combine_block(uint32_t fwd_addr, uint32_t bwd_addr, int lane, uint32_t (&pk)[16]) {
+__device__ __forceinline__ void combine_block(uint32_t fwd_addr, uint32_t bwd_addr, int lane, uint32_t masks, uint32_t (&pk)[16]) {
     if (REL != 0) {
         uint32_t r[32];
         tmem_ld32(REL < 0 ? fwd_addr : bwd_addr, r);
         tc_wait_ld();
 #pragma unroll
         for (int e = 0; e < 16; ++e) pk[e] = pack_bf16(as_f(r[2 * e]), as_f(r[2 * e + 1]));
-    } else {
+    } else if (masks == 0) {
+        // no mask table (a kernel without the shared memory for it): the same block by selects in fp32
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             uint32_t f[16], b[16];
@@ -102,27 +125,41 @@ __device__ __forceinline__ void combine_block(uint32_t fwd_addr, uint32_t bwd_ad
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const int s0 = 16 * h + 2 * e, s1 = s0 + 1;
-                // forward below the diagonal, backward above it, their sum on it (written as selects: it compiles to
-                // fewer instructions than masking both terms and adding them)
                 const float f0 = as_f(f[2 * e]), b0 = as_f(b[2 * e]), f1 = as_f(f[2 * e + 1]), b1 = as_f(b[2 * e + 1]);
                 const float lo = s0 < lane ? f0 : (s0 > lane ? b0 : f0 + b0);
                 const float hi = s1 < lane ? f1 : (s1 > lane ? b1 : f1 + b1);
                 pk[8 * h + e] = pack_bf16(lo, hi);
             }
         }
+    } else {
+        const uint32_t mrow = masks + (uint32_t)(((lane & 1) * 31 + 15 - (lane >> 1)) * 8);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            uint32_t f[16], b[16];
+            tmem_ld16(fwd_addr + 16 * h, f);
+            tmem_ld16(bwd_addr + 16 * h, b);
+            tc_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                uint32_t mf, mb;
+                asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(mf), "=r"(mb) : "r"(mrow + (uint32_t)(8 * h + e) * 8));
+                const uint32_t pf = pack_bf16(as_f(f[2 * e]), as_f(f[2 * e + 1])), pb = pack_bf16(as_f(b[2 * e]), as_f(b[2 * e + 1]));
+                pk[8 * h + e] = fma_bf16x2(pf, mf, mul_bf16x2(pb, mb));
+            }
+        }
     }
 }
 __device__ __forceinline__ void combine_any(int cb, int wq, bool valid, uint32_t fwd_addr, uint32_t bwd_addr, int lane,
-                                            uint32_t (&pk)[16]) {
+                                            uint32_t masks, uint32_t (&pk)[16]) {
     if (!valid) {
 #pragma unroll
         for (int e = 0; e < 16; ++e) pk[e] = 0u;
     } else if (cb < wq) {
-        combine_block<-1>(fwd_addr, bwd_addr, lane, pk);
+        combine_block<-1>(fwd_addr, bwd_addr, lane, masks, pk);
     } else if (cb == wq) {
-        combine_block<0>(fwd_addr, bwd_addr, lane, pk);
+        combine_block<0>(fwd_addr, bwd_addr, lane, masks, pk);
     } else {
-        combine_block<1>(fwd_addr, bwd_addr, lane, pk);
+        combine_block<1>(fwd_addr, bwd_addr, lane, masks, pk);
     }
 }
 
