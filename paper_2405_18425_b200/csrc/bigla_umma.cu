@@ -226,6 +226,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         for (int i = 0; i < 5; ++i) mbar_init(bar_g + 8 * i, 1);
         mbar_init(bar_pfx, 1);
         mbar_init(bar_g + 80, 1);   // never completed: only the test hook waits on it
+        mbar_init(bar_g + 88, 2);   // both chunks' summary batches are done (one phase per unit)
         *time_flag = 0;
         *early_gates = -1;
         *unit_slow_slot = 0;
@@ -520,20 +521,6 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 wait_mma();
             }
             if (nc == 2 && !SEG) {
-                if (ctl_warp && has_next) {
-                    // The summaries were the last readers of the k~ pair (chunk 1's batch included): the next unit's
-                    // log gates go there now, a good two microseconds before they are needed.
-                    bool go = false;
-                    if (elect_one()) {
-                        wait_bar(bar_mma + 8, (it * (uint32_t)(npass_c1 + 2) + (uint32_t)npass_c1) & 1);
-                        go = (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0;
-                        if (go) {
-                            load_gates(unit + ngroups, pair_qk);
-                            *early_gates = (int)it + 1;   // seen by every warp after the exchange barrier
-                        }
-                    }
-                    if (__any_sync(0xffffffffu, go)) next_gates_issued = true;
-                }
                 if (warp == 1 || warp == 4) {
                     // rows (TMEM lanes) 0..31 of U hold k~<^T v, rows 32..63 hold k~>^T v; lane = key dim.
                     // warp 1 (chunk 0, lanes 32..63): forward state for chunk 1; warp 4 (chunk 1, lanes 0..31): backward state
@@ -555,6 +542,19 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         }
                     }
                     fence_async_smem();
+                }
+                // Each chunk's issuing warp reports its summary batch done (its own wait above) on a barrier of its own: a
+                // parity wait on the other chunk's batch barrier could not tell which of that chunk's batches it sees.
+                if (issue_warp && elect_one()) mbar_arrive(bar_g + 88);
+                if (warp == 5 && has_next && elect_one()) {
+                    // The summaries were the last readers of the k~ pair: the next unit's log gates go there now, a good
+                    // two microseconds before they are needed.  Issued from chunk 1's issuing warp, which has no share in
+                    // the state hand-over that both chunks wait for.
+                    wait_bar(bar_g + 88, par);
+                    if ((slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3]) == 0 && *time_flag == 0) {
+                        load_gates(unit + ngroups, pair_qk);
+                        *early_gates = (int)it + 1;   // seen by every warp after the exchange barrier
+                    }
                 }
             }
         }
@@ -802,7 +802,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (nc == 2) wait_bar(bar_mma + 8, ((it + 1) * (uint32_t)(npass_c1 + 2) - 1) & 1);
                     go = (SEG ? *unit_slow_slot : (slow_slot[0] | slow_slot[1] | slow_slot[2] | slow_slot[3])) == 0 && *time_flag == 0;
                     if (go) {
-                        if (!next_gates_issued) load_gates(unit + ngroups, pair_qk);
+                        if (!(nc == 2 && !SEG && *early_gates == (int)it + 1)) load_gates(unit + ngroups, pair_qk);   // not on their way yet
                         load_qk(unit + ngroups, pair_g);
                     }
                 }
@@ -858,7 +858,7 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (elect_one()) {
                     tma_store_3d(&tm_o, 0, r0, unit, t_v);   // rows >= L and columns >= dv are clipped
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    if (has_next && !next_gates_issued) load_gates(unit + ngroups, pair_qk);
+                    if (has_next && !next_gates_issued && !(nc == 2 && !SEG && *early_gates == (int)it + 1)) load_gates(unit + ngroups, pair_qk);
                     if (has_next && !next_loads_issued) load_qk(unit + ngroups, pair_g);
                 }
                 next_gates_issued = next_loads_issued = false;
