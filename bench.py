@@ -281,6 +281,29 @@ def _summary(per_step_ms):
             "repeats": int(a.size)}
 
 
+def run_profile(args, cfg):
+    """A handful of launches of one call sequence over the rotating sets, for a profiler to capture."""
+    import torch
+
+    import paper_2405_18425_b200 as vig
+
+    torch.cuda.set_device(0)
+    lib = vig.load()
+    w = _Workload(cfg, lib, torch, torch.cuda.current_stream())
+    fn = {"fused": w.fused, "unfused": w.unfused, "scan": w.scan}[args.profile]
+    if args.profile == "scan":
+        w.unfused(0)   # log alpha of set 0 in place; the other sets' log alpha buffers hold arbitrary finite values
+        for d in w.sets[1:]:
+            d["la_f"].copy_(w.sets[0]["la_f"])
+            d["la_b"].copy_(w.sets[0]["la_b"])
+    torch.cuda.synchronize()
+    for i in range(args.warmup + args.steps):
+        fn(i)
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    print(json.dumps({"profile": args.profile, "workload": cfg.name, "launch_sequences": args.warmup + args.steps}))
+
+
 def run_gpu(args, cfg):
     import torch
 
@@ -387,7 +410,8 @@ def run_gpu(args, cfg):
     torch.cuda.empty_cache()
     if world == 1 and not args.only_headline:
         k_small = min(args.steps, 1000)
-        for other in [c for c in synth.CONFIGS if c.dtype == "bf16" and c.name != cfg.name]:
+        pool = synth.CONFIGS + (synth.SWEEP_CONFIGS if args.sweep else ())
+        for other in [c for c in pool if c.dtype == "bf16" and c.name != cfg.name]:
             wo = _Workload(other, lib, torch, stream)
             f_ms, _, _ = wo.time(wo.fused, k_small, args.warmup, 10.0)
             u_ms, _, _ = wo.time(wo.unfused, k_small, args.warmup, 10.0)
@@ -419,13 +443,19 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[c.name for c in synth.CONFIGS if c.dtype == "bf16"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=[c.name for c in synth.CONFIGS + synth.SWEEP_CONFIGS if c.dtype == "bf16"])
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--only-headline", action="store_true", help="skip the shorter runs of the other bf16 workloads")
+    ap.add_argument("--sweep", action="store_true",
+                    help="also time the second workload (resolution sweep, hierarchical stage shapes) in the `workloads` object")
+    ap.add_argument("--profile", choices=["fused", "unfused", "scan"],
+                    help="for profilers: W warm-up and K steps of one call sequence only, nothing else is launched or timed")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     cfg = synth.CONFIG_BY_NAME[args.workload]
-    if args.impl == "reference":
+    if args.profile:
+        run_profile(args, cfg)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_gpu(args, cfg)
