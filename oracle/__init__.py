@@ -9,4 +9,5 @@ from .oracle import (  # noqa: F401
     build_oracle,
     gate_prep,
 )
+from .locality import dwconv3x3, gate_blend  # noqa: F401
 from .quadratic import bigla_quadratic  # noqa: F401

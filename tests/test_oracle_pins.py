@@ -313,3 +313,110 @@ def test_gate_prep_matches_literal_definition(oracle):
         exact = mpmath.log(1 / (1 + mpmath.exp(-mpmath.mpf(gx)))) / 16
         got = oracle.gate_prep(np.array([gx]), 16.0)[0]
         assert abs(got - float(exact)) <= 4e-16 * abs(float(exact))
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 7: depth-wise 3x3 convolution and the 2-D gate blend (oracle/locality.py)
+# ----------------------------------------------------------------------------------------------
+
+def _pins_dwconv(conv):
+    from scipy import ndimage
+
+    r = np.random.default_rng(70)
+    x = r.standard_normal((2, 5, 7, 3))
+    w = r.standard_normal((3, 3, 3))
+    b = r.standard_normal(3)
+    got = conv(x, w, b)
+    # a library routine on the special case of one image and one channel: zero-padded cross-correlation
+    for n in range(2):
+        for c in range(3):
+            ref = ndimage.correlate(x[n, :, :, c], w[c], mode="constant", cval=0.0) + b[c]
+            np.testing.assert_allclose(got[n, :, :, c], ref, rtol=1e-13, atol=1e-13)
+    # brute force, tap by tap
+    for (n, i, j, c) in [(0, 0, 0, 0), (1, 4, 6, 2), (0, 2, 3, 1), (1, 0, 6, 0)]:
+        acc = b[c]
+        for di in (-1, 0, 1):
+            for dj in (-1, 0, 1):
+                if 0 <= i + di < 5 and 0 <= j + dj < 7:
+                    acc += w[c, di + 1, dj + 1] * x[n, i + di, j + dj, c]
+        assert abs(got[n, i, j, c] - acc) < 1e-13
+    # the centre tap alone is the identity; the tap above the centre reads the row above (zero at the top border)
+    delta = np.zeros((3, 3, 3)); delta[:, 1, 1] = 1.0
+    np.testing.assert_array_equal(conv(x, delta, None), x)
+    up = np.zeros((3, 3, 3)); up[:, 0, 1] = 1.0
+    s = conv(x, up, None)
+    np.testing.assert_array_equal(s[:, 1:], x[:, :-1])
+    np.testing.assert_array_equal(s[:, 0], 0.0)
+    left = np.zeros((3, 3, 3)); left[:, 1, 0] = 1.0
+    s = conv(x, left, None)
+    np.testing.assert_array_equal(s[:, :, 1:], x[:, :, :-1])
+    np.testing.assert_array_equal(s[:, :, 0], 0.0)
+    # zero padding: ones * ones counts the neighbours inside the grid (4 in a corner, 6 on an edge, 9 inside)
+    cnt = conv(np.ones((1, 4, 5, 1)), np.ones((1, 3, 3)), None)[0, :, :, 0]
+    assert cnt[0, 0] == 4 and cnt[0, 2] == 6 and cnt[2, 0] == 6 and cnt[2, 2] == 9 and cnt[3, 4] == 4
+    # depth-wise: a channel sees only its own filter and its own input; linear in x
+    x2 = x.copy(); x2[..., 1] += 5.0
+    d = conv(x2, w, b) - got
+    assert np.abs(d[..., 0]).max() == 0 and np.abs(d[..., 2]).max() == 0 and np.abs(d[..., 1]).max() > 0
+    np.testing.assert_allclose(conv(2.0 * x, w, None), 2.0 * conv(x, w, None), rtol=1e-13)
+    # a 1 x 1 grid keeps only the centre tap
+    one = conv(np.full((1, 1, 1, 2), 3.0), np.arange(18.0).reshape(2, 3, 3), np.array([1.0, -1.0]))
+    np.testing.assert_allclose(one[0, 0, 0], [3.0 * 4.0 + 1.0, 3.0 * 13.0 - 1.0])
+
+
+def _pins_blend(blend):
+    r = np.random.default_rng(71)
+    a, c = r.standard_normal((3, 4)), r.standard_normal((3, 4))
+    np.testing.assert_allclose(blend(a, np.zeros((3, 4)), c), 0.5 * (a + c), rtol=1e-15)
+    np.testing.assert_allclose(blend(a, np.full((3, 4), 50.0), c), a, rtol=1e-15, atol=1e-15)      # gate open: the local branch
+    np.testing.assert_allclose(blend(a, np.full((3, 4), -50.0), c), c, rtol=1e-15, atol=1e-15)     # gate closed: the global branch
+    assert np.isfinite(blend(a, np.full((3, 4), 800.0), c)).all() and np.isfinite(blend(a, np.full((3, 4), -800.0), c)).all()
+    z = r.standard_normal((3, 4)) * 3
+    np.testing.assert_allclose(blend(a, z, a), a, rtol=1e-15)                                   # the weights sum to one
+    # sigmoid(z) + sigmoid(-z) = 1: swapping the branches and negating z changes nothing
+    np.testing.assert_allclose(blend(a, z, c), blend(c, -z, a), rtol=1e-14)
+    mpmath.mp.dps = 50
+    for zz in (-7.5, -0.3, 0.0, 1.25, 11.0):
+        g = mpmath.mpf(1) / (1 + mpmath.e ** (-mpmath.mpf(zz)))
+        ref = g * mpmath.mpf(2) + (1 - g) * mpmath.mpf(-3)
+        assert abs(blend(np.array([2.0]), np.array([zz]), np.array([-3.0]))[0] - float(ref)) < 1e-15
+
+
+def test_dwconv_and_blend_oracle_pins():
+    from oracle.locality import dwconv3x3, gate_blend
+
+    _pins_dwconv(dwconv3x3)
+    _pins_blend(gate_blend)
+
+
+def test_planted_mistakes_in_eq7_are_caught():
+    from oracle.locality import dwconv3x3, gate_blend
+
+    def flipped(x, w, b):                     # a true convolution (kernel flipped) instead of the cross-correlation
+        return dwconv3x3(x, w[:, ::-1, ::-1], b)
+
+    def replicate(x, w, b):                   # edge replication instead of zero padding
+        xp = np.pad(np.asarray(x, dtype=np.float64), ((0, 0), (1, 1), (1, 1), (0, 0)), mode="edge")
+        out = np.zeros_like(np.asarray(x, dtype=np.float64))
+        for di in range(3):
+            for dj in range(3):
+                out += np.asarray(w)[None, None, None, :, di, dj] * xp[:, di:di + x.shape[1], dj:dj + x.shape[2], :]
+        return out + (0 if b is None else np.asarray(b)[None, None, None, :])
+
+    def shared_filter(x, w, b):               # one filter for every channel (not depth-wise)
+        return dwconv3x3(x, np.broadcast_to(np.asarray(w)[:1], np.asarray(w).shape), b)
+
+    for wrong in (flipped, replicate, shared_filter):
+        with pytest.raises(AssertionError):
+            _pins_dwconv(wrong)
+
+    def swapped(a, z, c):                     # the gate on the global branch
+        return gate_blend(c, z, a)
+
+    def tanh_gate(a, z, c):                   # a different squashing function
+        g = 0.5 * (1 + np.tanh(z))
+        return g * a + (1 - g) * c
+
+    for wrong in (swapped, tanh_gate):
+        with pytest.raises(AssertionError):
+            _pins_blend(wrong)
