@@ -16,6 +16,9 @@ from .binding import (  # noqa: F401
     vig_bigla_fwd_bf16,
     vig_bigla_fwd_f32,
     vig_bigla_fwd_gates_bf16,
+    vig_bigla_fwd_blend_bf16,
+    vig_dwconv3x3,
+    vig_gate_blend,
     vig_bigla_fwd_host,
     vig_bigla_fwd_static_bf16,
     vig_bigla_fwd_ws_bf16,

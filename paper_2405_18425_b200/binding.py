@@ -51,6 +51,14 @@ def load() -> ctypes.CDLL:
             getattr(lib, name).restype = ci
         lib.vig_bigla_fwd_gates_bf16.argtypes = [vp] * 6 + [ci] * 5 + [cf, vp]
         lib.vig_bigla_fwd_gates_bf16.restype = ci
+        lib.vig_bigla_fwd_blend_bf16.argtypes = [vp] * 8 + [ci] * 5 + [cf, vp]
+        lib.vig_bigla_fwd_blend_bf16.restype = ci
+        for name in ("vig_dwconv3x3_bf16", "vig_dwconv3x3_f32"):
+            getattr(lib, name).argtypes = [vp] * 4 + [ci] * 4 + [vp]
+            getattr(lib, name).restype = ci
+        for name in ("vig_gate_blend_bf16", "vig_gate_blend_f32"):
+            getattr(lib, name).argtypes = [vp] * 4 + [ctypes.c_longlong, vp]
+            getattr(lib, name).restype = ci
         lib.vig_bigla_fwd_host.argtypes = [vp] * 6 + [ci] * 5 + [cf, ci, vp]
         lib.vig_bigla_fwd_host.restype = ci
         lib.vig_status_string.argtypes = [ci]
@@ -164,6 +172,42 @@ def vig_bigla_fwd_gates_bf16(q, k, v, g_fwd, g_bwd, out, tau=16.0, stream=None):
     _check(load().vig_bigla_fwd_gates_bf16(q.data_ptr(), k.data_ptr(), v.data_ptr(), g_fwd.data_ptr(), g_bwd.data_ptr(),
                                            out.data_ptr(), *_dims(q, v), float(tau), _stream(stream)),
            "vig_bigla_fwd_gates_bf16")
+    return out
+
+
+def vig_bigla_fwd_blend_bf16(q, k, v, g_fwd, g_bwd, o_local, gate2d_logits, out, tau=16.0, stream=None):
+    """Forward pass from the gate logits with the 2-D gate blend of Eq. 7 in the same call."""
+    _dev(q, k, v, g_fwd, g_bwd, o_local, gate2d_logits, out)
+    _check(load().vig_bigla_fwd_blend_bf16(q.data_ptr(), k.data_ptr(), v.data_ptr(), g_fwd.data_ptr(), g_bwd.data_ptr(),
+                                           o_local.data_ptr(), gate2d_logits.data_ptr(), out.data_ptr(), *_dims(q, v),
+                                           float(tau), _stream(stream)), "vig_bigla_fwd_blend_bf16")
+    return out
+
+
+def _by_dtype(t, stem):
+    if t.dtype == torch.bfloat16:
+        return stem + "_bf16"
+    if t.dtype == torch.float32:
+        return stem + "_f32"
+    raise ValueError("bf16 or fp32 tensors only")
+
+
+def vig_dwconv3x3(x, w, bias, out, stream=None):
+    """Depth-wise 3x3 convolution (Eq. 7 line 1); x, out: [B, Hh, Ww, C]; w: [C, 3, 3]; bias: [C] or None."""
+    _dev(x, w, out)
+    name = _by_dtype(x, "vig_dwconv3x3")
+    B, Hh, Ww, C = x.shape
+    _check(getattr(load(), name)(x.data_ptr(), w.data_ptr(), bias.data_ptr() if bias is not None else None, out.data_ptr(),
+                                 B, Hh, Ww, C, _stream(stream)), name)
+    return out
+
+
+def vig_gate_blend(o_local, gate2d_logits, o_global, out, stream=None):
+    """out = sigmoid(z) * o_local + (1 - sigmoid(z)) * o_global, element-wise (Eq. 7 lines 3-4)."""
+    _dev(o_local, gate2d_logits, o_global, out)
+    name = _by_dtype(out, "vig_gate_blend")
+    _check(getattr(load(), name)(o_local.data_ptr(), gate2d_logits.data_ptr(), o_global.data_ptr(), out.data_ptr(),
+                                 out.numel(), _stream(stream)), name)
     return out
 
 

@@ -61,7 +61,7 @@ size_t tc_workspace_bytes(long long units, int L, int dk, int dv) {
 cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                             const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
                             int L, int dk, int dv, void* ws, cudaStream_t stream) {
-    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, 0.f, stream);
+    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, 0.f, nullptr, nullptr, stream);
     if (use_segments(units, L, dk, dv)) return launch_bigla_umma_seg(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
     return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
 }
@@ -148,11 +148,16 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
 // Forward pass from the gate logits (Eq. 5 line 1 + Eq. 6).  Units of at most 256 tokens on the tensor-core shapes:
 // one kernel that prepares log alpha on chip.  Everything else: gate preparation into scratch of the stream, then the
 // ordinary forward pass.
+// o_local != NULL: followed by the 2-D gate blend of Eq. 7 lines 3-4 (in the kernel's epilogue where one block covers a
+// unit, as an element-wise launch over `out` otherwise).
 static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, const void* g_f, const void* g_b, void* out,
-                               int B, int H, int L, int dk, int dv, float tau, cudaStream_t stream) {
+                               int B, int H, int L, int dk, int dv, float tau, const void* o_local, const void* z2d,
+                               cudaStream_t stream) {
     bool empty;
     int st = check_fwd_args(q, k, v, g_f, g_b, out, B, H, L, dk, dv, &empty);
     if (st != VIG_OK) return st;
+    if ((o_local != nullptr) != (z2d != nullptr)) return VIG_ERR_NULL_POINTER;
+    if (o_local && (!aligned16(o_local) || !aligned16(z2d))) return VIG_ERR_MISALIGNED;
     if (!(tau > 0.f) || !std::isfinite(tau)) return VIG_ERR_BAD_DIM;
     if (!tc_supported(dk, dv) && !recurrence_supported(dk, dv)) return VIG_ERR_UNSUPPORTED;
     if (empty) return VIG_OK;
@@ -160,7 +165,7 @@ static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, cons
     using bf = __nv_bfloat16;
     if (tc_supported(dk, dv) && umma_supported(dk, dv, L) && kernel_preference() == VIG_TEST_KERNEL_AUTO) {
         cudaError_t e = launch_bigla_umma((const bf*)q, (const bf*)k, (const bf*)v, (const bf*)g_f, (const bf*)g_b, (bf*)out,
-                                          units, L, dk, dv, tau, stream);
+                                          units, L, dk, dv, tau, (const bf*)o_local, (const bf*)z2d, stream);
         return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
     }
     const size_t n = (size_t)units * L * dk;
@@ -170,7 +175,29 @@ static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, cons
     st = vig_gate_prep_bf16(g_f, g_b, la, la + gate_bytes, B, H, L, dk, tau, stream);
     if (st == VIG_OK) st = vig_bigla_fwd_bf16(q, k, v, la, la + gate_bytes, out, B, H, L, dk, dv, stream);
     if (cudaFreeAsync(la, stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
+    if (st == VIG_OK && o_local &&
+        launch_gate_blend<bf>((const bf*)o_local, (const bf*)z2d, (const bf*)out, (bf*)out, (long long)units * L * dv, stream) != cudaSuccess)
+        st = VIG_ERR_CUDA;
     return st;
+}
+
+template <typename T>
+static int dwconv_impl(const void* x, const void* w, const void* bias, void* out, int B, int Hh, int Ww, int C, cudaStream_t stream) {
+    if (!x || !w || !out) return VIG_ERR_NULL_POINTER;
+    if (B < 0 || Hh < 0 || Ww < 0 || C < 1) return VIG_ERR_BAD_DIM;
+    if (!aligned16(x) || !aligned16(out)) return VIG_ERR_MISALIGNED;
+    if (!dwconv_supported(C, sizeof(T))) return VIG_ERR_UNSUPPORTED;
+    if (B == 0 || Hh == 0 || Ww == 0) return VIG_OK;
+    return launch_dwconv3x3<T>((const T*)x, (const T*)w, (const T*)bias, (T*)out, B, Hh, Ww, C, stream) == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
+template <typename T>
+static int blend_impl(const void* o_local, const void* z, const void* o_global, void* out, long long n, cudaStream_t stream) {
+    if (!o_local || !z || !o_global || !out) return VIG_ERR_NULL_POINTER;
+    if (n < 0) return VIG_ERR_BAD_DIM;
+    if (!aligned16(o_local) || !aligned16(z) || !aligned16(o_global) || !aligned16(out)) return VIG_ERR_MISALIGNED;
+    if (n == 0) return VIG_OK;
+    return launch_gate_blend<T>((const T*)o_local, (const T*)z, (const T*)o_global, (T*)out, n, stream) == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
 }
 
 static int fwd_f32_impl(const void* q, const void* k, const void* v, const void* la_f, const void* la_b, void* out,
@@ -260,7 +287,27 @@ int vig_bigla_fwd_f32(const void* q, const void* k, const void* v, const void* l
 
 int vig_bigla_fwd_gates_bf16(const void* q, const void* k, const void* v, const void* g_fwd, const void* g_bwd, void* out,
                              int B, int H, int L, int dk, int dv, float tau, void* stream) {
-    return fwd_gates_bf16_impl(q, k, v, g_fwd, g_bwd, out, B, H, L, dk, dv, tau, (cudaStream_t)stream);
+    return fwd_gates_bf16_impl(q, k, v, g_fwd, g_bwd, out, B, H, L, dk, dv, tau, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+int vig_bigla_fwd_blend_bf16(const void* q, const void* k, const void* v, const void* g_fwd, const void* g_bwd,
+                             const void* o_local, const void* gate2d_logits, void* out, int B, int H, int L, int dk, int dv,
+                             float tau, void* stream) {
+    if (!o_local || !gate2d_logits) return VIG_ERR_NULL_POINTER;
+    return fwd_gates_bf16_impl(q, k, v, g_fwd, g_bwd, out, B, H, L, dk, dv, tau, o_local, gate2d_logits, (cudaStream_t)stream);
+}
+
+int vig_dwconv3x3_bf16(const void* x, const void* w, const void* bias, void* out, int B, int Hh, int Ww, int C, void* stream) {
+    return dwconv_impl<__nv_bfloat16>(x, w, bias, out, B, Hh, Ww, C, (cudaStream_t)stream);
+}
+int vig_dwconv3x3_f32(const void* x, const void* w, const void* bias, void* out, int B, int Hh, int Ww, int C, void* stream) {
+    return dwconv_impl<float>(x, w, bias, out, B, Hh, Ww, C, (cudaStream_t)stream);
+}
+int vig_gate_blend_bf16(const void* o_local, const void* gate2d_logits, const void* o_global, void* out, long long n, void* stream) {
+    return blend_impl<__nv_bfloat16>(o_local, gate2d_logits, o_global, out, n, (cudaStream_t)stream);
+}
+int vig_gate_blend_f32(const void* o_local, const void* gate2d_logits, const void* o_global, void* out, long long n, void* stream) {
+    return blend_impl<float>(o_local, gate2d_logits, o_global, out, n, (cudaStream_t)stream);
 }
 
 size_t vig_bigla_workspace_bytes(int B, int H, int L, int dk, int dv, int dtype) {

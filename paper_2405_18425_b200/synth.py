@@ -180,3 +180,16 @@ def make_inputs(cfg: BiglaConfig, units: slice | None = None) -> dict:
         "g_fwd": store(g_f, cfg.dtype).reshape(shape_k),
         "g_bwd": store(g_b, cfg.dtype).reshape(shape_k),
     }
+
+
+def make_locality_inputs(cfg: BiglaConfig, units: slice | None = None) -> dict:
+    """Stored O_local and 2-D gate logits z of the locality injection (Eq. 7), [B, H, L, dv] like v and out: streams 5
+    and 6 of the configuration's seed, both N(0, 1) (stand-ins for the depth-wise convolution's output laid out per
+    head and for its projection O_local W + b).  `units` as in make_inputs."""
+    lo, hi, _ = (units or slice(None)).indices(cfg.units)
+    count, first = (hi - lo) * cfg.L * cfg.dv, lo * cfg.L * cfg.dv
+    shape = (cfg.B, cfg.H, cfg.L, cfg.dv) if units is None else (hi - lo, 1, cfg.L, cfg.dv)
+    return {
+        "o_local": store(standard_normal(cfg.seed, 5, count, first), cfg.dtype).reshape(shape),
+        "z2d": store(standard_normal(cfg.seed, 6, count, first), cfg.dtype).reshape(shape),
+    }
