@@ -212,6 +212,12 @@ class _Workload:
                 # a cheap re-draw for the extra sets: a rotation of the flattened tensor keeps the value
                 # distribution and the [B,H,L,d] structure-free i.i.d. statistics of the generator
                 d[n] = t if s == 0 else torch.roll(t.flatten(), 7919 * s).view_as(t).contiguous()
+            if s == 0:
+                loc = synth.make_locality_inputs(cfg)
+                d["o_local"], d["z2d"] = (torch.from_numpy(loc[n].view(np.int16)).cuda().view(torch.bfloat16) for n in ("o_local", "z2d"))
+            else:   # the blend's two extra inputs of the other sets: rotations of set 0's, like the other tensors
+                d["o_local"] = torch.roll(self.sets[0]["o_local"].flatten(), 7919 * s).view_as(d["v"]).contiguous()
+                d["z2d"] = torch.roll(self.sets[0]["z2d"].flatten(), 7919 * s).view_as(d["v"]).contiguous()
             d["la_f"] = torch.empty_like(d["g_fwd"])
             d["la_b"] = torch.empty_like(d["g_bwd"])
             d["out"] = torch.empty_like(d["v"])
@@ -226,7 +232,10 @@ class _Workload:
                    d["out"].data_ptr(), cfg.B, cfg.H, cfg.L, cfg.dk, cfg.dv, sp)
             fused = (d["q"].data_ptr(), d["k"].data_ptr(), d["v"].data_ptr(), d["g_fwd"].data_ptr(), d["g_bwd"].data_ptr(),
                      d["out"].data_ptr(), cfg.B, cfg.H, cfg.L, cfg.dk, cfg.dv, float(cfg.tau), sp)
-            self.calls.append((gate, fwd, fused))
+            blend = (d["q"].data_ptr(), d["k"].data_ptr(), d["v"].data_ptr(), d["g_fwd"].data_ptr(), d["g_bwd"].data_ptr(),
+                     d["o_local"].data_ptr(), d["z2d"].data_ptr(), d["out"].data_ptr(), cfg.B, cfg.H, cfg.L, cfg.dk, cfg.dv,
+                     float(cfg.tau), sp)
+            self.calls.append((gate, fwd, fused, blend))
 
     # one step of each kind on buffer set i
     def fused(self, i):
@@ -234,9 +243,13 @@ class _Workload:
             raise RuntimeError("vig_bigla_fwd_gates_bf16 failed")
 
     def unfused(self, i):
-        gate, fwd, _ = self.calls[i % self.n_sets]
+        gate, fwd = self.calls[i % self.n_sets][:2]
         if (self.lib.vig_gate_prep_bf16(*gate) | self.lib.vig_bigla_fwd_bf16(*fwd)) != 0:
             raise RuntimeError("vig_gate_prep_bf16 + vig_bigla_fwd_bf16 failed")
+
+    def blend(self, i):
+        if self.lib.vig_bigla_fwd_blend_bf16(*self.calls[i % self.n_sets][3]) != 0:
+            raise RuntimeError("vig_bigla_fwd_blend_bf16 failed")
 
     def scan(self, i):
         if self.lib.vig_bigla_fwd_bf16(*self.calls[i % self.n_sets][1]) != 0:
@@ -346,6 +359,7 @@ def run_gpu(args, cfg):
     clocks = sampler.summary(t_host0, t_host1)
     unfused_ms, _, _ = w.time(w.unfused, args.steps, args.warmup, 20.0, dist, vdist)   # also leaves log alpha in place for the scan
     scan_ms, _, _ = w.time(w.scan, min(args.steps, 2000), args.warmup, 20.0, dist, vdist)
+    blend_ms, _, _ = w.time(w.blend, min(args.steps, 2000), args.warmup, 20.0, dist, vdist)
     assert vig.vig_last_device_status() == 0, "a device-side bounded wait expired"
     ms_per_step = float(np.median(step_ms))
     scan_us = float(np.median(scan_ms)) * 1e3
@@ -372,6 +386,11 @@ def run_gpu(args, cfg):
         "clocks": clocks, "gpu_launches": int(launches),
     }
     line["roofline_step"]["traffic"] = None   # no capture of the fused kernel yet
+    # the layer's call with the 2-D gate blend of the locality injection in the epilogue: two more [B,H,L,dv] inputs
+    blend_bytes = cfg.algorithmic_bytes + 2 * cfg.units * cfg.L * cfg.dv * cfg.elem_bytes
+    blend_us = float(np.median(blend_ms)) * 1e3
+    line["blend_step"] = dict(_summary(blend_ms), step="vig_bigla_fwd_blend_bf16", algorithmic_bytes=blend_bytes,
+                              achieved_gbs=blend_bytes / (blend_us * 1e-6) / 1e9, frac=blend_bytes / (blend_us * 1e-6) / 1e9 / peak)
 
     if rank == 0:
         # ---- end to end through the host-buffer entry point (H2D + kernels + D2H in the timed region) ----

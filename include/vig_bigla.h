@@ -159,8 +159,11 @@ int vig_bigla_fwd_gates_bf16(const void* q, const void* k, const void* v,
  * vig_dwconv3x3_*: depth-wise 3 x 3 convolution over the patch grid (Eq. 7 line 1), stride 1, zero padding 1,
  * cross-correlation (the convention of deep-learning convolutions: w[c][0][1] weighs the pixel above).
  * x, out: [B, Hh, Ww, C] channels last (the mixer's sequence is the row-major Hh x Ww grid); w: [C, 3, 3];
- * bias: [C] or NULL; all of the call's element type; fp32 accumulation.  C must be a multiple of 8 (bf16) or
- * 4 (fp32), at most 5120.  x and out must not overlap.  Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED, CUDA. */
+ * bias: [C] or NULL; all of the call's element type and 16-byte aligned; fp32 accumulation.  C must be a multiple of
+ * 8 (bf16) or 4 (fp32), at most 2^20.  x and out must not overlap.  The input tiles (with the padding, which reads
+ * outside the image supply as zeros) come by tiled TMA loads; a load that never completes ends the kernel's bounded
+ * wait and shows up as VIG_ERR_DEVICE_TIMEOUT in vig_last_device_status.
+ * Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED, CUDA. */
 int vig_dwconv3x3_bf16(const void* x, const void* w, const void* bias, void* out,
                        int B, int Hh, int Ww, int C, void* stream);
 int vig_dwconv3x3_f32(const void* x, const void* w, const void* bias, void* out,
@@ -175,10 +178,8 @@ int vig_gate_blend_f32(const void* o_local, const void* gate2d_logits, const voi
 /* vig_bigla_fwd_blend_bf16: vig_bigla_fwd_gates_bf16 followed by the blend, in one call (Eq. 5 line 1, Eq. 6 and
  * Eq. 7 lines 3-4): out = G * o_local + (1 - G) * BiGLA(q, k, v, logsigmoid(g_fwd)/tau, logsigmoid(g_bwd)/tau).
  * o_local, gate2d_logits: [B,H,L,dv] like out (the caller lays the channels of O_local and of O_local W + b out per
- * head).  Units of at most 256 tokens on the tensor-core head sizes blend in the epilogue of the forward kernel
- * (each thread reads its token's rows of the two tensors; the gate through the hardware tanh, absolute error about
- * 5e-4 on a weight whose result is rounded to bf16); other shapes run the forward call, then vig_gate_blend_bf16 over
- * `out`.  Errors: as vig_bigla_fwd_gates_bf16. */
+ * head).  The blend runs as an element-wise launch over `out` behind the forward launch(es), in the same stream (it finds
+ * `out` in L2; sigmoid in fp32).  Errors: as vig_bigla_fwd_gates_bf16. */
 int vig_bigla_fwd_blend_bf16(const void* q, const void* k, const void* v,
                              const void* g_fwd, const void* g_bwd,
                              const void* o_local, const void* gate2d_logits, void* out,

@@ -61,7 +61,7 @@ size_t tc_workspace_bytes(long long units, int L, int dk, int dv) {
 cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                             const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
                             int L, int dk, int dv, void* ws, cudaStream_t stream) {
-    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, 0.f, nullptr, nullptr, stream);
+    if (umma_supported(dk, dv, L)) return launch_bigla_umma(q, k, v, la_f, la_b, out, units, L, dk, dv, 0.f, stream);
     if (use_segments(units, L, dk, dv)) return launch_bigla_umma_seg(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
     return launch_bigla_umma_long(q, k, v, la_f, la_b, out, units, L, dk, dv, ws, stream);
 }
@@ -148,8 +148,10 @@ static int fwd_bf16_impl(const void* q, const void* k, const void* v, const void
 // Forward pass from the gate logits (Eq. 5 line 1 + Eq. 6).  Units of at most 256 tokens on the tensor-core shapes:
 // one kernel that prepares log alpha on chip.  Everything else: gate preparation into scratch of the stream, then the
 // ordinary forward pass.
-// o_local != NULL: followed by the 2-D gate blend of Eq. 7 lines 3-4 (in the kernel's epilogue where one block covers a
-// unit, as an element-wise launch over `out` otherwise).
+// o_local != NULL: followed by the 2-D gate blend of Eq. 7 lines 3-4 as an element-wise launch over `out` (programmatic
+// dependent launch: its set-up overlaps the forward kernel's tail, and it finds `out` in L2).  The blend inside the forward
+// kernel's epilogue was built and measured slower than this chain: the forward kernel is bound by the dependent chain
+// of a unit, two units per SM, and whatever the epilogue adds lengthens that chain.
 static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, const void* g_f, const void* g_b, void* out,
                                int B, int H, int L, int dk, int dv, float tau, const void* o_local, const void* z2d,
                                cudaStream_t stream) {
@@ -165,7 +167,9 @@ static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, cons
     using bf = __nv_bfloat16;
     if (tc_supported(dk, dv) && umma_supported(dk, dv, L) && kernel_preference() == VIG_TEST_KERNEL_AUTO) {
         cudaError_t e = launch_bigla_umma((const bf*)q, (const bf*)k, (const bf*)v, (const bf*)g_f, (const bf*)g_b, (bf*)out,
-                                          units, L, dk, dv, tau, (const bf*)o_local, (const bf*)z2d, stream);
+                                          units, L, dk, dv, tau, stream);
+        if (e == cudaSuccess && o_local)
+            e = launch_gate_blend<bf>((const bf*)o_local, (const bf*)z2d, (const bf*)out, (bf*)out, (long long)units * L * dv, stream);
         return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
     }
     const size_t n = (size_t)units * L * dk;
@@ -185,8 +189,8 @@ template <typename T>
 static int dwconv_impl(const void* x, const void* w, const void* bias, void* out, int B, int Hh, int Ww, int C, cudaStream_t stream) {
     if (!x || !w || !out) return VIG_ERR_NULL_POINTER;
     if (B < 0 || Hh < 0 || Ww < 0 || C < 1) return VIG_ERR_BAD_DIM;
-    if (!aligned16(x) || !aligned16(out)) return VIG_ERR_MISALIGNED;
-    if (!dwconv_supported(C, sizeof(T))) return VIG_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(out) || !aligned16(w) || (bias && !aligned16(bias))) return VIG_ERR_MISALIGNED;
+    if (!dwconv_supported(C, sizeof(T)) || (long long)B * Hh * Ww > 0x7fffffffLL) return VIG_ERR_UNSUPPORTED;
     if (B == 0 || Hh == 0 || Ww == 0) return VIG_OK;
     return launch_dwconv3x3<T>((const T*)x, (const T*)w, (const T*)bias, (T*)out, B, Hh, Ww, C, stream) == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
 }

@@ -92,18 +92,7 @@ struct UArgs {
     // fused gate preparation only (GATES): la_f / la_b hold the gate logits g, and log alpha = logsigmoid(g) / tau
     float inv_tau;
     int expire_wait;   // test hook: every block lets one bounded wait, on an mbarrier nothing completes, run out
-    // 2-D gate blend in the epilogue only (BLEND, Eq. 7 lines 3-4): out = G o_local + (1 - G) BiGLA(..), G = sigmoid(z2d);
-    // both [units][L][DV] like out
-    const __nv_bfloat16 *o_local, *z2d;
 };
-
-// sigmoid(z) = (1 + tanh(z / 2)) / 2 with the hardware tanh (absolute error about 5e-4: the weight of a blend whose
-// result is rounded to bf16)
-__device__ __forceinline__ float sigmoid_fast(float z) {
-    float t;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * z));
-    return fmaf(0.5f, t, 0.5f);
-}
 
 // log2 alpha = logsigmoid(g) / (tau ln 2) (Eq. 5 line 1, in base 2 so that the operand scaling needs no further
 // multiplication) for the eight bf16 gate logits of one 16-byte piece, evaluated in fp32 as
@@ -146,14 +135,13 @@ __device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned l
     asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
-template <int DK, int DV, bool SEG, bool GATES, bool BLEND>
+template <int DK, int DV, bool SEG, bool GATES>
 __global__ void __launch_bounds__(kThreads, 2)
 bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_f, const __grid_constant__ CUtensorMap tm_b,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, const UArgs args) {
     static_assert((DK == 16 || DK == 24 || DK == 32) && (DV == 32 || DV == 48 || DV == 64), "unsupported head size");
     static_assert(!(SEG && GATES), "fused gate preparation is built for the single-block form only");
-    static_assert(!BLEND || GATES, "the blend epilogue comes with fused gate preparation (the layer's call)");
     extern __shared__ __align__(1024) uint8_t smem_raw[];   // the swizzled tiles need the 1 KB alignment; no slack is allocated
     const uint32_t base = smem_u32(smem_raw);
     uint8_t* bp = smem_raw;
@@ -838,27 +826,12 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     else asm volatile("bar.arrive 6, 160;" ::: "memory");
                 }
                 if (row_live) {
-                    // (BLEND) this token's rows of O_local and of the 2-D gate logits, straight from global memory
-                    const size_t grow = BLEND ? ((size_t)unit * args.L + row) * DV : 0;
 #pragma unroll
                     for (int ch = 0; ch < DV / 8; ++ch) {
                         uint32_t o[4];
-                        if constexpr (BLEND) {
-                            // Eq. 7 lines 3-4: O = G O_local + (1 - G) O_global, O_global = (P v + q~ S_in) / 2, in fp32
-                            const uint4 l4 = __ldg(reinterpret_cast<const uint4*>(args.o_local + grow + ch * 8));
-                            const uint4 z4 = __ldg(reinterpret_cast<const uint4*>(args.z2d + grow + ch * 8));
-                            const uint32_t lw[4] = {l4.x, l4.y, l4.z, l4.w}, zw[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const float2 lo = unpack_bf16(lw[e]), zz = unpack_bf16(zw[e]);
-                                const float g0 = 0.5f * as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e]), g1 = 0.5f * as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e + 1]);
-                                o[e] = pack_bf16(fmaf(sigmoid_fast(zz.x), lo.x - g0, g0), fmaf(sigmoid_fast(zz.y), lo.y - g1, g1));
-                            }
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 4; ++e)   // halved after packing: exact (a power of two), one instruction per pair
-                                o[e] = mul_bf16x2(pack_bf16(as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e]), as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e + 1])), 0x3F003F00u);
-                        }
+                        for (int e = 0; e < 4; ++e)   // halved after packing: exact (a power of two), one instruction per pair
+                            o[e] = mul_bf16x2(pack_bf16(as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e]), as_f(r[ch >> 2][(ch & 3) * 8 + 2 * e + 1])), 0x3F003F00u);
                         *reinterpret_cast<uint4*>(bp + lay.v + sw_off<128>(row, ch)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
@@ -927,20 +900,20 @@ bigla_umma_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 struct DevPlan {
     int sms, per_sm;
 };
-template <int DK, int DV, bool SEG, bool GATES, bool BLEND>
+template <int DK, int DV, bool SEG, bool GATES>
 cudaError_t device_plan(size_t smem_max, DevPlan* out) {
     static std::atomic<int> sms_of[kMaxDevices], per_sm_of[kMaxDevices];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
     int sms = sms_of[dev].load(std::memory_order_acquire);
     if (sms == 0) {
-        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV, SEG, GATES, BLEND>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
+        cudaError_t e = cudaFuncSetAttribute(bigla_umma_kernel<DK, DV, SEG, GATES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
         if (e != cudaSuccess) return e;
         // Blocks of this kernel an SM holds at once, from the resources themselves: two (2 x 256 of the 512 TMEM columns)
         // if shared memory (plus the kilobyte the system keeps per block) and the register file admit them.  The occupancy
         // calculator of the runtime reports one block for this kernel where the hardware runs two.
         cudaFuncAttributes fa;
-        if ((e = cudaFuncGetAttributes(&fa, bigla_umma_kernel<DK, DV, SEG, GATES, BLEND>)) != cudaSuccess) return e;
+        if ((e = cudaFuncGetAttributes(&fa, bigla_umma_kernel<DK, DV, SEG, GATES>)) != cudaSuccess) return e;
         int smem_sm = 0, regs_sm = 0;
         if ((e = cudaDeviceGetAttribute(&smem_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&regs_sm, cudaDevAttrMaxRegistersPerMultiprocessor, dev)) != cudaSuccess) return e;
@@ -955,12 +928,11 @@ cudaError_t device_plan(size_t smem_max, DevPlan* out) {
     return cudaSuccess;
 }
 
-// GATES: la_f / la_b are the gate logits and `tau` their temperature (fused gate preparation).  BLEND: o_local and z2d
-// feed the 2-D gate blend of the epilogue.
-template <int DK, int DV, bool GATES, bool BLEND>
+// GATES: la_f / la_b are the gate logits and `tau` their temperature (fused gate preparation).
+template <int DK, int DV, bool GATES>
 cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                           const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units, int L,
-                          float tau, const __nv_bfloat16* o_local, const __nv_bfloat16* z2d, cudaStream_t stream) {
+                          float tau, cudaStream_t stream) {
     const int rows = (L + 15) / 16 * 16;
     CUtensorMap tq, tk, tf, tb, tv, to;
     if (!make_map(&tq, q, units, L, DK, 32, rows) || !make_map(&tk, k, units, L, DK, 32, rows) ||
@@ -971,8 +943,6 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     a.q = q; a.k = k; a.v = v; a.la_f = la_f; a.la_b = la_b; a.out = out; a.L = L; a.rows = rows; a.units = units;
     a.nseg = 1;
     a.inv_tau = GATES ? 1.f / tau : 0.f;
-    a.o_local = o_local;
-    a.z2d = z2d;
     a.expire_wait = take_expire_next_wait();
     a.dev_status = device_status_ptr();
     if (!a.dev_status) return cudaErrorUnknown;
@@ -984,13 +954,13 @@ cudaError_t launch_umma_t(const __nv_bfloat16* q, const __nv_bfloat16* k, const 
     size_t most = make_layout(kMaxRows, false).total;
     if (most < rec) most = rec;
     DevPlan dp;
-    cudaError_t e = device_plan<DK, DV, false, GATES, BLEND>(most, &dp);
+    cudaError_t e = device_plan<DK, DV, false, GATES>(most, &dp);
     if (e != cudaSuccess) return e;
     // Persistent blocks, two per SM: block b takes units b, b + grid, b + 2 grid, ...  (Nothing waits for another block
     // here, so a grid larger than what is resident at once only costs time.)
     const long long cap = 2LL * dp.sms;
     const long long grid = units < cap ? units : cap;
-    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV, false, GATES, BLEND>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV, false, GATES>, dim3((unsigned)grid), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
     count_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
 }
@@ -1025,13 +995,13 @@ cudaError_t launch_umma_seg_t(const __nv_bfloat16* q, const __nv_bfloat16* k, co
     const size_t rec = (size_t)rec_plan(kThreads, DK, DV).smem_floats * 4;
     if (smem < rec) smem = rec;
     DevPlan dp;
-    cudaError_t e = device_plan<DK, DV, true, false, false>(smem, &dp);
+    cudaError_t e = device_plan<DK, DV, true, false>(smem, &dp);
     if (e != cudaSuccess) return e;
     const long long cap = (long long)dp.per_sm * dp.sms;
     long long groups = cap / nseg;
     if (groups < 1) return cudaErrorLaunchOutOfResources;
     if (groups > units) groups = units;
-    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV, true, false, false>, dim3((unsigned)(groups * nseg)), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
+    const cudaError_t le = launch_pdl(bigla_umma_kernel<DK, DV, true, false>, dim3((unsigned)(groups * nseg)), dim3(kThreads), smem, stream, tq, tk, tf, tb, tv, to, a);
     count_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
 }
@@ -1065,15 +1035,11 @@ cudaError_t launch_bigla_umma_seg(const __nv_bfloat16* q, const __nv_bfloat16* k
 
 cudaError_t launch_bigla_umma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                               const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out, long long units,
-                              int L, int dk, int dv, float gate_tau, const __nv_bfloat16* o_local, const __nv_bfloat16* z2d,
-                              cudaStream_t stream) {
-    if (o_local && !(gate_tau > 0.f)) return cudaErrorInvalidValue;   // the blend epilogue comes with fused gate preparation
-#define VIG_CASE(DK_, DV_)                                                                                                        \
-    if (dk == DK_ && dv == DV_) {                                                                                                 \
-        if (o_local) return launch_umma_t<DK_, DV_, true, true>(q, k, v, la_f, la_b, out, units, L, gate_tau, o_local, z2d, stream); \
-        return gate_tau > 0.f ? launch_umma_t<DK_, DV_, true, false>(q, k, v, la_f, la_b, out, units, L, gate_tau, nullptr, nullptr, stream) \
-                              : launch_umma_t<DK_, DV_, false, false>(q, k, v, la_f, la_b, out, units, L, 0.f, nullptr, nullptr, stream);   \
-    }
+                              int L, int dk, int dv, float gate_tau, cudaStream_t stream) {
+#define VIG_CASE(DK_, DV_)                                                                                              \
+    if (dk == DK_ && dv == DV_)                                                                                         \
+        return gate_tau > 0.f ? launch_umma_t<DK_, DV_, true>(q, k, v, la_f, la_b, out, units, L, gate_tau, stream)     \
+                              : launch_umma_t<DK_, DV_, false>(q, k, v, la_f, la_b, out, units, L, 0.f, stream);
     VIG_CASE(16, 32) VIG_CASE(16, 48) VIG_CASE(16, 64)
     VIG_CASE(24, 32) VIG_CASE(24, 48) VIG_CASE(24, 64)
     VIG_CASE(32, 32) VIG_CASE(32, 48) VIG_CASE(32, 64)

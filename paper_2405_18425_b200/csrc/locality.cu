@@ -5,6 +5,7 @@
 #include <atomic>
 
 #include "ptx.cuh"
+#include "tma_host.h"
 #include "vig_internal.h"
 
 namespace vig {
@@ -12,14 +13,14 @@ namespace vig {
 namespace {
 
 template <typename T>
-struct Vec;   // 16 bytes of T as fp32 lanes
+struct Vec;   // 16 bytes of T: Raw as loaded, N fp32 lanes unpacked
 template <>
 struct Vec<float> {
     static constexpr int N = 4;
-    static __device__ __forceinline__ void load(const float* p, float (&f)[4]) {
-        const float4 v = *reinterpret_cast<const float4*>(p);
-        f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
-    }
+    using Raw = float4;
+    static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    static __device__ __forceinline__ void unpack(const Raw& v, float (&f)[4]) { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
+    static __device__ __forceinline__ void load(const float* p, float (&f)[4]) { unpack(*reinterpret_cast<const float4*>(p), f); }
     static __device__ __forceinline__ void store(float* p, const float (&f)[4]) {
         *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
     }
@@ -27,8 +28,9 @@ struct Vec<float> {
 template <>
 struct Vec<__nv_bfloat16> {
     static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) {
-        const uint4 v = *reinterpret_cast<const uint4*>(p);
+    using Raw = uint4;
+    static __device__ __forceinline__ Raw zero() { return make_uint4(0u, 0u, 0u, 0u); }
+    static __device__ __forceinline__ void unpack(const Raw& v, float (&f)[8]) {
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int x = 0; x < 4; ++x) {
@@ -37,6 +39,7 @@ struct Vec<__nv_bfloat16> {
             f[2 * x + 1] = t.y;
         }
     }
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) { unpack(*reinterpret_cast<const uint4*>(p), f); }
     static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&f)[8]) {
         *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
     }
@@ -45,45 +48,109 @@ struct Vec<__nv_bfloat16> {
 __device__ __forceinline__ float to_f(float x) { return x; }
 __device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
 
-// Thread = one pixel x one group of V channels (16 bytes).  The filters sit in shared memory as fp32, tap major
-// ([9][C]), so that the V channels of a tap are one or two 16-byte reads; the nine neighbours come through L1 / L2 (each
-// input line is used by the nine pixels around it).  fp32 accumulation, zero padding, cross-correlation:
+// Depth-wise 3 x 3 convolution, fp32 accumulation, zero padding, cross-correlation:
 //   out[n, i, j, c] = b[c] + sum_{di, dj} w[c, di + 1, dj + 1] x[n, i + di, j + dj, c].
+// Task = th output rows x tw columns of one image for one slab of gpb channel groups (a group = 16 bytes of channels).  Its
+// input tile with the one-pixel halo, (th + 2) x (tw + 2) x gpb groups, comes by ONE tiled TMA load, which also supplies
+// the zero padding (coordinates outside the image read as zero) - the bytes in flight occupy no registers, and an
+// input element crosses L2 once per tile that needs it instead of nine times.  A block keeps its slab (blockIdx.y) and
+// strides over tasks with two tile buffers: the next tile loads while this one is worked on.
+// Thread = one channel group of one column: its V filters (nine taps each, 144 contiguous bytes of w) and biases sit
+// in registers as fp32; walking down the tile it reads three 16-byte pieces per input row (left, centre, right) from
+// shared memory and adds them into the three output rows they touch, which live in rolling accumulators.  Lanes run
+// over channel groups first, so shared-memory reads and the 16-byte output stores are contiguous per warp.
 template <typename T>
-__global__ void __launch_bounds__(256) dwconv3x3_kernel(const T* __restrict__ x, const T* __restrict__ w, const T* __restrict__ bias,
-                                                        T* __restrict__ out, long long pixels, int Hh, int Ww, int C) {
+__global__ void __launch_bounds__(256) dwconv3x3_kernel(const __grid_constant__ CUtensorMap tm_x, const T* __restrict__ w,
+                                                        const T* __restrict__ bias, T* __restrict__ out, int Hh, int Ww, int C, int gpb, int tw,
+                                                        int th, int rowsegs, int coltiles, int tasks, int* dev_status) {
     constexpr int V = Vec<T>::N;
-    extern __shared__ __align__(16) float wsm[];   // [9][C] then the bias [C]
+    using Raw = typename Vec<T>::Raw;
+    extern __shared__ __align__(128) uint8_t dw_smem[];
+    __shared__ __align__(8) unsigned long long dw_bar[2];
+    const uint32_t tile_bytes = (uint32_t)(th + 2) * (tw + 2) * gpb * 16;
+    const uint32_t buf_pitch = (tile_bytes + 127) / 128 * 128;
+    const uint32_t bar0 = smem_u32(dw_bar);
     pdl_launch_dependents();
-    pdl_wait();
-    for (int e = threadIdx.x; e < 9 * C; e += blockDim.x) {
-        const int c = e / 9, tap = e - 9 * c;
-        wsm[tap * C + c] = to_f(w[e]);
+    if (threadIdx.x == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int c = threadIdx.x; c < C; c += blockDim.x) wsm[9 * C + c] = bias ? to_f(bias[c]) : 0.f;
     __syncthreads();
-    const int groups = C / V;
-    const long long total = pixels * groups;
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
-        const long long pix = idx / groups;
-        const int c0 = (int)(idx - pix * groups) * V;
-        const int j = (int)(pix % Ww), i = (int)((pix / Ww) % Hh);
-        float acc[V];
+    const int col = threadIdx.x / gpb, g = threadIdx.x % gpb;
+    const int c_slab = blockIdx.y * gpb * V, c0 = c_slab + g * V;
+    const bool chan_live = c0 < C;   // ragged last slab
+    auto issue = [&](int task, int buf) {   // one thread: the tile of `task` into buffer `buf`
+        const int j0 = (task % coltiles) * tw, i0 = ((task / coltiles) % rowsegs) * th, n = task / (coltiles * rowsegs);
+        mbar_expect_tx(bar0 + 8 * buf, tile_bytes);
+        tma_load_4d(smem_u32(dw_smem) + buf * buf_pitch, &tm_x, c_slab, j0 - 1, i0 - 1, n, bar0 + 8 * buf);
+    };
+    pdl_wait();   // x may be the output of the kernel before this one in the stream
+    if (threadIdx.x == 0 && (int)blockIdx.x < tasks) issue(blockIdx.x, 0);
+    float wr[9][V], br[V];
 #pragma unroll
-        for (int u = 0; u < V; ++u) acc[u] = wsm[9 * C + c0 + u];
+    for (int u = 0; u < V; ++u) br[u] = 0.f;
+    if (chan_live) {
+        float t[9 * V];   // w[c0 .. c0 + V)[3][3]: 9 V contiguous elements = nine 16-byte pieces
 #pragma unroll
-        for (int di = -1; di <= 1; ++di) {
+        for (int x9 = 0; x9 < 9; ++x9) {
+            float f[V];
+            Vec<T>::load(w + (size_t)c0 * 9 + x9 * V, f);
 #pragma unroll
-            for (int dj = -1; dj <= 1; ++dj) {
-                if (i + di < 0 || i + di >= Hh || j + dj < 0 || j + dj >= Ww) continue;   // zero padding
-                float xv[V];
-                Vec<T>::load(x + ((pix + (long long)di * Ww + dj) * C + c0), xv);
-                const float* wt = wsm + ((di + 1) * 3 + (dj + 1)) * C + c0;
+            for (int u = 0; u < V; ++u) t[x9 * V + u] = f[u];
+        }
 #pragma unroll
-                for (int u = 0; u < V; ++u) acc[u] = fmaf(wt[u], xv[u], acc[u]);
+        for (int tap = 0; tap < 9; ++tap)
+#pragma unroll
+            for (int u = 0; u < V; ++u) wr[tap][u] = t[u * 9 + tap];
+        if (bias) Vec<T>::load(bias + c0, br);
+    }
+    const uint32_t row_pitch_s = (uint32_t)(tw + 2) * gpb * 16;   // one tile row in shared memory
+    const size_t row_pitch_g = (size_t)Ww * C;
+    int it = 0;
+    for (int task = blockIdx.x; task < tasks; task += gridDim.x, ++it) {
+        const int buf = it & 1;
+        // (every thread has left the other buffer: the barrier that ended the previous round)
+        if (threadIdx.x == 0 && task + (int)gridDim.x < tasks) issue(task + gridDim.x, buf ^ 1);
+        const bool arrived = mbar_wait_bounded(bar0 + 8 * buf, (it >> 1) & 1);
+        if (!__syncthreads_and(arrived)) {   // a load that never lands: report it and leave, all threads together
+            if (threadIdx.x == 0) atomicOr(dev_status, kDevStatusTimeout);
+            break;
+        }
+        const int j0 = (task % coltiles) * tw, i0 = ((task / coltiles) % rowsegs) * th, n = task / (coltiles * rowsegs);
+        const int j = j0 + col, rows = min(th, Hh - i0);   // output rows i0 .. i0 + rows - 1
+        if (chan_live && j < Ww) {
+            const uint8_t* tp = dw_smem + buf * buf_pitch + ((uint32_t)col * gpb + g) * 16;   // tile row 0, column j - 1
+            T* op = out + (((size_t)n * Hh + i0) * Ww + j) * C + c0;
+            // a_up: the output row above the input row at hand (complete with it), a_mid: the one at it, a_dn: the one below
+            float a_up[V], a_mid[V];
+#pragma unroll
+            for (int u = 0; u < V; ++u) a_up[u] = a_mid[u] = br[u];
+            for (int r = 0; r < rows + 2; ++r) {   // tile row r = input row i0 - 1 + r (zeros outside the image)
+                float in[3][V];
+#pragma unroll
+                for (int d = 0; d < 3; ++d)
+                    Vec<T>::unpack(*reinterpret_cast<const Raw*>(tp + (uint32_t)r * row_pitch_s + (uint32_t)d * gpb * 16), in[d]);
+                float a_dn[V];
+#pragma unroll
+                for (int u = 0; u < V; ++u) {
+                    a_dn[u] = br[u];
+#pragma unroll
+                    for (int d = 0; d < 3; ++d) {
+                        a_up[u] = fmaf(wr[6 + d][u], in[d][u], a_up[u]);
+                        a_mid[u] = fmaf(wr[3 + d][u], in[d][u], a_mid[u]);
+                        a_dn[u] = fmaf(wr[d][u], in[d][u], a_dn[u]);
+                    }
+                }
+                if (r >= 2) Vec<T>::store(op + (size_t)(r - 2) * row_pitch_g, a_up);
+#pragma unroll
+                for (int u = 0; u < V; ++u) {
+                    a_up[u] = a_mid[u];
+                    a_mid[u] = a_dn[u];
+                }
             }
         }
-        Vec<T>::store(out + (pix * C + c0), acc);
+        __syncthreads();   // the tile may be overwritten by the load after next
     }
 }
 
@@ -133,22 +200,39 @@ cudaError_t sm_count(int* sms) {
 
 }  // namespace
 
-bool dwconv_supported(int C, size_t elem) { return C >= 1 && C % (int)(16 / elem) == 0 && (size_t)10 * C * 4 <= 200 * 1024; }
+bool dwconv_supported(int C, size_t elem) { return C >= 1 && C % (int)(16 / elem) == 0 && C <= (1 << 20); }
 
 template <typename T>
 cudaError_t launch_dwconv3x3(const T* x, const T* w, const T* bias, T* out, long long images, int Hh, int Ww, int C, cudaStream_t stream) {
     int sms = 0;
     cudaError_t e = sm_count(&sms);
     if (e != cudaSuccess) return e;
-    const size_t smem = (size_t)10 * C * sizeof(float);
-    if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(dwconv3x3_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
+    constexpr int V = (int)(16 / sizeof(T));
+    const int groups = C / V;
+    const int slabs = (groups + 15) / 16, gpb = (groups + slabs - 1) / slabs;   // channel groups per block: at most 16
+    const int coltiles = (Ww + 256 / gpb - 1) / (256 / gpb), tw = (Ww + coltiles - 1) / coltiles;   // at most 256 threads, 256 columns
+    const int rowsegs = (Hh + 7) / 8, th = (Hh + rowsegs - 1) / rowsegs;                            // at most 8 output rows per tile
+    const long long tasks = images * rowsegs * coltiles;
+    if (tasks > 0x7fffffffLL || slabs > 65535 || tw + 2 > 256) return cudaErrorInvalidValue;
+    const size_t tile = (size_t)(th + 2) * (tw + 2) * gpb * 16, smem = 2 * ((tile + 127) / 128 * 128);
+    if (smem > 200 * 1024) return cudaErrorInvalidValue;
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!configured[dev].load(std::memory_order_acquire)) {
+        if ((e = cudaFuncSetAttribute(dwconv3x3_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess) return e;
+        configured[dev].store(true, std::memory_order_release);
     }
-    const long long pixels = images * Hh * Ww, work = pixels * (C / (int)(16 / sizeof(T)));
-    long long blocks = (work + 255) / 256;
-    if (blocks > 8LL * sms) blocks = 8LL * sms;
-    const cudaError_t le = launch_pdl(dwconv3x3_kernel<T>, dim3((unsigned)blocks), dim3(256), smem, stream, x, w, bias, out, pixels, Hh, Ww, C);
+    CUtensorMap tm;
+    if (!make_map_nhwc(&tm, x, images, Hh, Ww, C, (int)sizeof(T), gpb * V, tw + 2, th + 2)) return cudaErrorInvalidValue;
+    int* status = device_status_ptr();
+    if (!status) return cudaErrorInvalidValue;
+    long long nb = 2LL * sms / slabs;   // two blocks per SM over all slabs
+    if (nb < 1) nb = 1;
+    if (nb > tasks) nb = tasks;
+    const cudaError_t le = launch_pdl(dwconv3x3_kernel<T>, dim3((unsigned)nb, (unsigned)slabs), dim3((unsigned)(tw * gpb)), smem, stream, tm, w,
+                                      bias, out, Hh, Ww, C, gpb, tw, th, rowsegs, coltiles, (int)tasks, status);
     count_launch();
     return le != cudaSuccess ? le : cudaGetLastError();
 }

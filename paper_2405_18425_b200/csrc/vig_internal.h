@@ -39,11 +39,9 @@ cudaError_t launch_bigla_tc(const __nv_bfloat16* q, const __nv_bfloat16* k, cons
 // ---- bf16 tcgen05 / TMEM path (units of at most 256 tokens) ----
 bool umma_supported(int dk, int dv, int L);
 // gate_tau > 0: la_f / la_b hold the gate logits g and the kernel prepares log alpha = logsigmoid(g) / gate_tau itself.
-// o_local != NULL (with gate_tau > 0): the epilogue blends, out = G o_local + (1 - G) BiGLA(..), G = sigmoid(z2d).
 cudaError_t launch_bigla_umma(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v,
                               const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
-                              long long units, int L, int dk, int dv, float gate_tau, const __nv_bfloat16* o_local,
-                              const __nv_bfloat16* z2d, cudaStream_t stream);
+                              long long units, int L, int dk, int dv, float gate_tau, cudaStream_t stream);
 
 // ---- Eq. 7 around the mixer: depth-wise 3 x 3 convolution (channels last) and the 2-D gate blend ----
 bool dwconv_supported(int C, size_t elem);

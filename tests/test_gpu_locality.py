@@ -104,6 +104,34 @@ def test_fused_blend_gate_limits(oracle):
     np.testing.assert_array_equal(got[..., 32:], device_to_f64(plain, "bf16")[..., 32:])
 
 
+def test_fused_blend_on_a_unit_handed_to_the_recurrence(oracle):
+    """A unit whose gates leave the range of the factorised tiles is evaluated by the recurrence inside the same launch;
+    its output must be blended like every other unit's."""
+    cfg, x = random_problem(3400, 2, 3, 196, 32, 64, "bf16")
+    g = synth.stored_to_f64(x["g_fwd"], "bf16").copy()
+    g[1, 1, 10:140] = -10.0            # log alpha = -10 / 16 per token: -80 over a chunk
+    x["g_fwd"] = synth.store(g, "bf16")
+    vig.vig_test_take_fallback_count()
+    got, ref = _run_blend(oracle, cfg, x, synth.make_locality_inputs(cfg))
+    assert vig.vig_test_take_fallback_count() == 1
+    assert rel_err(got[1, 1], ref[1, 1]) <= TOL["bf16"]
+    assert rel_err(got, ref) <= TOL["bf16"]
+
+
+def test_dwconv3x3_many_channels_in_slabs(oracle):
+    """More than 256 sixteen-byte channel groups: the groups are split over the grid's second dimension, raggedly."""
+    rng = np.random.default_rng(77)
+    B, Hh, Ww, C = 1, 5, 6, 2056
+    x = synth.store(rng.standard_normal((B, Hh, Ww, C)), "bf16")
+    w = synth.store(rng.standard_normal((C, 3, 3)) / 3, "bf16")
+    b = synth.store(rng.standard_normal(C), "bf16")
+    out = torch.full((B, Hh, Ww, C), float("nan"), device="cuda", dtype=torch.bfloat16)
+    vig.vig_dwconv3x3(to_device(x, "bf16"), to_device(w, "bf16"), to_device(b, "bf16"), out)
+    f = lambda a: synth.stored_to_f64(a, "bf16")
+    ref = oracle.dwconv3x3(f(x), f(w), f(b))
+    assert rel_err(device_to_f64(out, "bf16"), ref) <= TOL["bf16"]
+
+
 def test_locality_entry_points_validate_arguments():
     lib = vig.load()
     buf = torch.empty(4096, device="cuda", dtype=torch.bfloat16)
