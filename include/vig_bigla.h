@@ -185,6 +185,28 @@ int vig_bigla_fwd_blend_bf16(const void* q, const void* k, const void* v,
                              const void* o_local, const void* gate2d_logits, void* out,
                              int B, int H, int L, int dk, int dv, float tau, void* stream);
 
+/* ---- Gradient of the forward pass ------------------------------------------------------------------------------
+ * The paper trains with the layer of Eq. 6 (its Appendix C gives the recipe) without describing the gradient; this is
+ * the reverse-mode adjoint of Eq. 6 as it stands.  For d_out = dLoss/d_out [B,H,L,dv] the call writes
+ *   dq, dk_out [B,H,L,dk], dv_out [B,H,L,dv], dlog_alpha_fwd, dlog_alpha_bwd [B,H,L,dk]
+ * (gradients with respect to the LOG gates as passed to the forward call; a caller that feeds gate logits g chains
+ * dg = dlog_alpha * (1 - sigmoid(g)) / tau, Eq. 5 line 1).  All device pointers of the call's element type, contiguous,
+ * 16-byte aligned; inputs are not written; outputs must not overlap inputs or one another.
+ * How: dv is the forward pass itself on (k, q, d_out) with the gates moved by one token (the tensor-core kernels for
+ * the bf16 head sizes they cover); dq, dk and the gate gradients come from two fp32 walks over the sequence per unit
+ * on the CUDA cores (states in registers), with the gate gradients as running sums of q * dq - k * dk per direction.
+ * Scratch (the moved gates, 8 L dk bytes per unit of partial results) comes from the library's pool, stream-ordered.
+ * Head sizes: dk <= 128, dv <= 128, and whatever the forward entry point of the same type takes.
+ * Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED, CUDA. */
+int vig_bigla_bwd_bf16(const void* q, const void* k, const void* v,
+                       const void* log_alpha_fwd, const void* log_alpha_bwd, const void* d_out,
+                       void* dq, void* dk_out, void* dv_out, void* dlog_alpha_fwd, void* dlog_alpha_bwd,
+                       int B, int H, int L, int dk, int dv, void* stream);
+int vig_bigla_bwd_f32(const void* q, const void* k, const void* v,
+                      const void* log_alpha_fwd, const void* log_alpha_bwd, const void* d_out,
+                      void* dq, void* dk_out, void* dv_out, void* dlog_alpha_fwd, void* dlog_alpha_bwd,
+                      int B, int H, int L, int dk, int dv, void* stream);
+
 /* ---- Whole path on HOST buffers -------------------------------------------------------------------
  * Gate preparation followed by the BiGLA forward (Eq. 5 line 1 + Eq. 6) for callers whose data
  * lives in host memory.  All seven pointers are HOST pointers (pinned memory makes the copies

@@ -17,6 +17,7 @@ from .binding import (  # noqa: F401
     vig_bigla_fwd_f32,
     vig_bigla_fwd_gates_bf16,
     vig_bigla_fwd_blend_bf16,
+    vig_bigla_bwd,
     vig_dwconv3x3,
     vig_gate_blend,
     vig_bigla_fwd_host,

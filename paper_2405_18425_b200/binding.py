@@ -59,6 +59,9 @@ def load() -> ctypes.CDLL:
         for name in ("vig_gate_blend_bf16", "vig_gate_blend_f32"):
             getattr(lib, name).argtypes = [vp] * 4 + [ctypes.c_longlong, vp]
             getattr(lib, name).restype = ci
+        for name in ("vig_bigla_bwd_bf16", "vig_bigla_bwd_f32"):
+            getattr(lib, name).argtypes = [vp] * 11 + [ci] * 5 + [vp]
+            getattr(lib, name).restype = ci
         lib.vig_bigla_fwd_host.argtypes = [vp] * 6 + [ci] * 5 + [cf, ci, vp]
         lib.vig_bigla_fwd_host.restype = ci
         lib.vig_status_string.argtypes = [ci]
@@ -190,6 +193,17 @@ def _by_dtype(t, stem):
     if t.dtype == torch.float32:
         return stem + "_f32"
     raise ValueError("bf16 or fp32 tensors only")
+
+
+def vig_bigla_bwd(q, k, v, log_alpha_fwd, log_alpha_bwd, d_out, dq, dk, dv, dlog_alpha_fwd, dlog_alpha_bwd, stream=None):
+    """Gradient of the forward pass (Eq. 6) for d_out = dLoss/d_out; writes and returns the five gradient tensors."""
+    ts = (q, k, v, log_alpha_fwd, log_alpha_bwd, d_out, dq, dk, dv, dlog_alpha_fwd, dlog_alpha_bwd)
+    _dev(*ts)
+    name = _by_dtype(q, "vig_bigla_bwd")
+    if any(t.dtype != q.dtype for t in ts):
+        raise ValueError("all tensors of one call share a dtype")
+    _check(getattr(load(), name)(*(t.data_ptr() for t in ts), *_dims(q, v), _stream(stream)), name)
+    return dq, dk, dv, dlog_alpha_fwd, dlog_alpha_bwd
 
 
 def vig_dwconv3x3(x, w, bias, out, stream=None):

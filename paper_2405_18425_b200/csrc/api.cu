@@ -185,6 +185,40 @@ static int fwd_gates_bf16_impl(const void* q, const void* k, const void* v, cons
     return st;
 }
 
+static int fwd_f32_impl(const void* q, const void* k, const void* v, const void* la_f, const void* la_b, void* out,
+                        int B, int H, int L, int dk, int dv, cudaStream_t stream);
+
+// Gradient of the forward pass (Eq. 6) for d_out = dLoss/d_out.  Three steps in the stream: the gates shifted by one
+// token, the forward pass on (k, q, d_out) with them (= dv), the two recurrence walks for dq, dk and the gate gradients.
+template <typename T>
+static int bwd_impl(const void* q, const void* k, const void* v, const void* la_f, const void* la_b, const void* d_out, void* dq,
+                    void* dk_out, void* dv_out, void* dla_f, void* dla_b, int B, int H, int L, int dk, int dv, cudaStream_t stream) {
+    bool empty;
+    int st = check_fwd_args(q, k, v, la_f, la_b, d_out, B, H, L, dk, dv, &empty);
+    if (st != VIG_OK) return st;
+    if (!dq || !dk_out || !dv_out || !dla_f || !dla_b) return VIG_ERR_NULL_POINTER;
+    if (!aligned16(dq) || !aligned16(dk_out) || !aligned16(dv_out) || !aligned16(dla_f) || !aligned16(dla_b)) return VIG_ERR_MISALIGNED;
+    if (!bwd_supported(dk, dv)) return VIG_ERR_UNSUPPORTED;
+    if (sizeof(T) == 2 ? !(tc_supported(dk, dv) || recurrence_supported(dk, dv)) : !recurrence_supported(dk, dv)) return VIG_ERR_UNSUPPORTED;
+    if (empty) return VIG_OK;
+    const long long units = (long long)B * H;
+    const size_t gate_bytes = ((size_t)units * L * dk * sizeof(T) + 255) / 256 * 256;
+    char* scratch = nullptr;
+    if (pool_alloc((void**)&scratch, 2 * gate_bytes + bwd_scratch_bytes(units, L, dk), stream) != cudaSuccess) return VIG_ERR_CUDA;
+    T *sf = (T*)scratch, *sb = (T*)(scratch + gate_bytes);
+    if (launch_shift_gates<T>((const T*)la_f, (const T*)la_b, sf, sb, units, L, dk, stream) != cudaSuccess) st = VIG_ERR_CUDA;
+    if (st == VIG_OK) {
+        if constexpr (sizeof(T) == 2) st = fwd_bf16_impl(k, q, d_out, sf, sb, dv_out, B, H, L, dk, dv, nullptr, 0, true, stream);
+        else st = fwd_f32_impl(k, q, d_out, sf, sb, dv_out, B, H, L, dk, dv, stream);
+    }
+    if (st == VIG_OK && launch_bigla_bwd<T>((const T*)q, (const T*)k, (const T*)v, (const T*)la_f, (const T*)la_b, (const T*)d_out, (T*)dq,
+                                            (T*)dk_out, (T*)dla_f, (T*)dla_b, (float*)(scratch + 2 * gate_bytes), units, L, dk, dv,
+                                            stream) != cudaSuccess)
+        st = VIG_ERR_CUDA;
+    if (cudaFreeAsync(scratch, stream) != cudaSuccess && st == VIG_OK) st = VIG_ERR_CUDA;
+    return st;
+}
+
 template <typename T>
 static int dwconv_impl(const void* x, const void* w, const void* bias, void* out, int B, int Hh, int Ww, int C, cudaStream_t stream) {
     if (!x || !w || !out) return VIG_ERR_NULL_POINTER;
@@ -299,6 +333,19 @@ int vig_bigla_fwd_blend_bf16(const void* q, const void* k, const void* v, const 
                              float tau, void* stream) {
     if (!o_local || !gate2d_logits) return VIG_ERR_NULL_POINTER;
     return fwd_gates_bf16_impl(q, k, v, g_fwd, g_bwd, out, B, H, L, dk, dv, tau, o_local, gate2d_logits, (cudaStream_t)stream);
+}
+
+int vig_bigla_bwd_bf16(const void* q, const void* k, const void* v, const void* log_alpha_fwd, const void* log_alpha_bwd,
+                       const void* d_out, void* dq, void* dk_out, void* dv_out, void* dlog_alpha_fwd, void* dlog_alpha_bwd, int B, int H,
+                       int L, int dk, int dv, void* stream) {
+    return bwd_impl<__nv_bfloat16>(q, k, v, log_alpha_fwd, log_alpha_bwd, d_out, dq, dk_out, dv_out, dlog_alpha_fwd, dlog_alpha_bwd, B, H, L,
+                                   dk, dv, (cudaStream_t)stream);
+}
+int vig_bigla_bwd_f32(const void* q, const void* k, const void* v, const void* log_alpha_fwd, const void* log_alpha_bwd,
+                      const void* d_out, void* dq, void* dk_out, void* dv_out, void* dlog_alpha_fwd, void* dlog_alpha_bwd, int B, int H,
+                      int L, int dk, int dv, void* stream) {
+    return bwd_impl<float>(q, k, v, log_alpha_fwd, log_alpha_bwd, d_out, dq, dk_out, dv_out, dlog_alpha_fwd, dlog_alpha_bwd, B, H, L, dk, dv,
+                           (cudaStream_t)stream);
 }
 
 int vig_dwconv3x3_bf16(const void* x, const void* w, const void* bias, void* out, int B, int Hh, int Ww, int C, void* stream) {

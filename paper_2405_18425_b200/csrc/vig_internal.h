@@ -65,6 +65,16 @@ cudaError_t launch_bigla_umma_long(const __nv_bfloat16* q, const __nv_bfloat16* 
                                    const __nv_bfloat16* la_f, const __nv_bfloat16* la_b, __nv_bfloat16* out,
                                    long long units, int L, int dk, int dv, void* ws, cudaStream_t stream);
 
+// ---- gradient of the forward pass with respect to q, k and the log gates (fp32 recurrences on the CUDA cores); the
+// gradient with respect to v is the forward pass on (k, q, d_out) with the gates from launch_shift_gates ----
+bool bwd_supported(int dk, int dv);
+size_t bwd_scratch_bytes(long long units, int L, int dk);
+template <typename T>
+cudaError_t launch_shift_gates(const T* la_f, const T* la_b, T* out_f, T* out_b, long long units, int L, int dk, cudaStream_t stream);
+template <typename T>
+cudaError_t launch_bigla_bwd(const T* q, const T* k, const T* v, const T* la_f, const T* la_b, const T* d_out, T* dq, T* dk_out, T* dla_f,
+                             T* dla_b, float* scratch, long long units, int L, int dk, int dv, cudaStream_t stream);
+
 // Launch with programmatic stream serialization: the kernel's prologue (everything before its pdl_wait) may overlap
 // the tail of the kernel before it in the stream.
 template <typename... KArgs, typename... Args>

@@ -193,3 +193,12 @@ def make_locality_inputs(cfg: BiglaConfig, units: slice | None = None) -> dict:
         "o_local": store(standard_normal(cfg.seed, 5, count, first), cfg.dtype).reshape(shape),
         "z2d": store(standard_normal(cfg.seed, 6, count, first), cfg.dtype).reshape(shape),
     }
+
+
+def make_grad_input(cfg: BiglaConfig, units: slice | None = None) -> np.ndarray:
+    """Stored d_out = dLoss/d_out of the gradient call, [B, H, L, dv] like out: stream 7 of the configuration's seed,
+    N(0, 1) (a stand-in for what the layers after the mixer send back).  `units` as in make_inputs."""
+    lo, hi, _ = (units or slice(None)).indices(cfg.units)
+    count, first = (hi - lo) * cfg.L * cfg.dv, lo * cfg.L * cfg.dv
+    shape = (cfg.B, cfg.H, cfg.L, cfg.dv) if units is None else (hi - lo, 1, cfg.L, cfg.dv)
+    return store(standard_normal(cfg.seed, 7, count, first), cfg.dtype).reshape(shape)

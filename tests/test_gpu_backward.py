@@ -1,0 +1,103 @@
+"""GPU parity of the gradient of the forward pass (vig_bigla_bwd_*) against the fp64 gradient oracle
+(oracle/backward.py) on the same seeded inputs.  Bars as for the forward pass, per gradient tensor:
+max|gpu - oracle| <= 1e-4 (fp32) / 2e-2 (bf16) of max|oracle|."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2405_18425_b200 as vig
+from paper_2405_18425_b200 import synth
+
+from helpers import TOL, device_to_f64, oracle_log_alpha, random_problem, rel_err, to_device, to_stored
+
+pytestmark = pytest.mark.gpu
+
+NAMES = ("dq", "dk", "dv", "dlog_alpha_fwd", "dlog_alpha_bwd")
+
+
+def _run(oracle, cfg, x, d_out, units=None):
+    """GPU gradient of the whole problem; the oracle on `units` (a slice of the flattened (b, h) units) or on all."""
+    la_f = oracle_log_alpha(oracle, x["g_fwd"], cfg.dtype, cfg.tau)
+    la_b = oracle_log_alpha(oracle, x["g_bwd"], cfg.dtype, cfg.tau)
+    host = dict(q=x["q"], k=x["k"], v=x["v"], f=la_f, b=la_b, g=d_out)
+    d = {n: to_device(a, cfg.dtype) for n, a in host.items()}
+    outs = [torch.full_like(d[n], float("nan")) for n in ("q", "k", "v", "f", "b")]
+    vig.vig_bigla_bwd(d["q"], d["k"], d["v"], d["f"], d["b"], d["g"], *outs)
+    torch.cuda.synchronize()
+    assert vig.vig_last_device_status() == 0
+    for n, a in host.items():   # inputs are never written
+        np.testing.assert_array_equal(to_stored(d[n], cfg.dtype), a)
+    sel = (lambda a: a) if units is None else (lambda a: a.reshape((-1, 1) + a.shape[2:])[units])
+    f = lambda a: synth.stored_to_f64(sel(a), cfg.dtype)
+    ref = oracle.bigla_bwd(f(x["q"]), f(x["k"]), f(x["v"]), f(la_f), f(la_b), f(d_out))
+    got = [sel(device_to_f64(o, cfg.dtype)) for o in outs]
+    return got, ref
+
+
+def _check(got, ref, dtype, label=""):
+    for name, g, r in zip(NAMES, got, ref):
+        assert np.isfinite(g).all(), name
+        err = rel_err(g, r)
+        if label:
+            print(f"observed {label} {name}: max|gpu-oracle|/max|oracle| = {err:.3e} (bar {TOL[dtype]:g})")
+        assert err <= TOL[dtype], (name, err)
+
+
+@pytest.mark.parametrize("dk,dv", [(16, 32), (24, 48), (32, 64), (8, 16), (40, 72), (64, 128)])
+@pytest.mark.parametrize("L", [1, 2, 15, 16, 17, 100, 196, 300])
+def test_bf16_gradient_small_and_ragged(oracle, dk, dv, L):
+    """Lengths below, at and across the sixteen-token staging, one and two tokens, head sizes on and off the
+    tensor-core path of the forward pass that supplies dv."""
+    cfg, x = random_problem(4000 + L, 2, 2, L, dk, dv, "bf16", gate_mean=1.0)
+    got, ref = _run(oracle, cfg, x, synth.make_grad_input(cfg))
+    _check(got, ref, "bf16")
+
+
+@pytest.mark.parametrize("dk,dv,L", [(16, 32, 7), (5, 3, 33), (32, 64, 130), (24, 48, 50), (3, 2, 6), (128, 128, 20)])
+def test_f32_gradient_shapes(oracle, dk, dv, L):
+    cfg, x = random_problem(4100 + L, 2, 2, L, dk, dv, "f32", gate_mean=0.5)
+    got, ref = _run(oracle, cfg, x, synth.make_grad_input(cfg))
+    _check(got, ref, "f32")
+
+
+def test_gradient_strong_gates(oracle):
+    """Gates far below one (log alpha down to about -1 per token): states die within a few tokens, the gate
+    gradients are sums of strongly cancelling terms."""
+    cfg, x = random_problem(4200, 2, 2, 150, 32, 64, "f32", gate_mean=-3.0, tau=4.0)
+    got, ref = _run(oracle, cfg, x, synth.make_grad_input(cfg))
+    _check(got, ref, "f32")
+
+
+@pytest.mark.parametrize("idx", [0, 1, 3, 4], ids=[synth.CONFIGS[i].name for i in (0, 1, 3, 4)])
+def test_gradient_benchmark_config_full_size(oracle, idx):
+    """Configurations at full size through the entry point the benchmark times; the oracle (which keeps every state of
+    the sequence) on a sample of units spread over the batch: units are independent."""
+    cfg = synth.CONFIGS[idx]
+    x, g = synth.make_inputs(cfg), synth.make_grad_input(cfg)
+    step = max(1, cfg.units // 6)
+    units = slice(0, cfg.units, step) if cfg.L <= 256 else slice(0, cfg.units, max(1, cfg.units // 2))
+    got, ref = _run(oracle, cfg, x, g, units)
+    _check(got, ref, cfg.dtype, cfg.name)
+
+
+def test_gradient_entry_point_validates_arguments():
+    lib = vig.load()
+    buf = torch.zeros(1 << 16, device="cuda", dtype=torch.bfloat16)
+    p = buf.data_ptr()
+    before = vig.vig_kernel_launch_count()
+    args = [p + 8192 * n for n in range(11)]   # eleven separate 4096-element regions
+    assert lib.vig_bigla_bwd_bf16(*args, 1, 1, 8, 16, 32, None) == 0
+    torch.cuda.synchronize()
+    launched = vig.vig_kernel_launch_count() - before
+    assert launched >= 3                                                        # gates moved, forward pass for dv, the walks
+    for missing in range(11):
+        a = list(args)
+        a[missing] = None
+        assert lib.vig_bigla_bwd_bf16(*a, 1, 1, 8, 16, 32, None) == -1
+    a = list(args)
+    a[7] = p + 2
+    assert lib.vig_bigla_bwd_bf16(*a, 1, 1, 8, 16, 32, None) == -4
+    assert lib.vig_bigla_bwd_bf16(*args, 1, -1, 8, 16, 32, None) == -2
+    assert lib.vig_bigla_bwd_bf16(*args, 1, 1, 8, 200, 32, None) == -3          # head size beyond the kernel's
+    assert lib.vig_bigla_bwd_bf16(*args, 0, 1, 8, 16, 32, None) == 0            # empty
+    assert vig.vig_kernel_launch_count() - before == launched
