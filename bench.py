@@ -218,6 +218,13 @@ class _Workload:
             else:   # the blend's two extra inputs of the other sets: rotations of set 0's, like the other tensors
                 d["o_local"] = torch.roll(self.sets[0]["o_local"].flatten(), 7919 * s).view_as(d["v"]).contiguous()
                 d["z2d"] = torch.roll(self.sets[0]["z2d"].flatten(), 7919 * s).view_as(d["v"]).contiguous()
+            # the gradient call: d_out in (stream 7 of the generator; rotations for the other sets), five gradients out
+            if s == 0:
+                d["d_out"] = torch.from_numpy(synth.make_grad_input(cfg).view(np.int16)).cuda().view(torch.bfloat16)
+            else:
+                d["d_out"] = torch.roll(self.sets[0]["d_out"].flatten(), 7919 * s).view_as(d["v"]).contiguous()
+            for n, like in (("dq", "q"), ("dk", "k"), ("dv", "v"), ("dla_f", "q"), ("dla_b", "q")):
+                d[n] = torch.empty_like(d[like])
             d["la_f"] = torch.empty_like(d["g_fwd"])
             d["la_b"] = torch.empty_like(d["g_bwd"])
             d["out"] = torch.empty_like(d["v"])
@@ -235,7 +242,10 @@ class _Workload:
             blend = (d["q"].data_ptr(), d["k"].data_ptr(), d["v"].data_ptr(), d["g_fwd"].data_ptr(), d["g_bwd"].data_ptr(),
                      d["o_local"].data_ptr(), d["z2d"].data_ptr(), d["out"].data_ptr(), cfg.B, cfg.H, cfg.L, cfg.dk, cfg.dv,
                      float(cfg.tau), sp)
-            self.calls.append((gate, fwd, fused, blend))
+            bwd = (d["q"].data_ptr(), d["k"].data_ptr(), d["v"].data_ptr(), d["la_f"].data_ptr(), d["la_b"].data_ptr(),
+                   d["d_out"].data_ptr(), d["dq"].data_ptr(), d["dk"].data_ptr(), d["dv"].data_ptr(), d["dla_f"].data_ptr(),
+                   d["dla_b"].data_ptr(), cfg.B, cfg.H, cfg.L, cfg.dk, cfg.dv, sp)
+            self.calls.append((gate, fwd, fused, blend, bwd))
 
     # one step of each kind on buffer set i
     def fused(self, i):
@@ -250,6 +260,10 @@ class _Workload:
     def blend(self, i):
         if self.lib.vig_bigla_fwd_blend_bf16(*self.calls[i % self.n_sets][3]) != 0:
             raise RuntimeError("vig_bigla_fwd_blend_bf16 failed")
+
+    def bwd(self, i):   # (log alpha of every set is in place once the un-fused step has run over the sets)
+        if self.lib.vig_bigla_bwd_bf16(*self.calls[i % self.n_sets][4]) != 0:
+            raise RuntimeError("vig_bigla_bwd_bf16 failed")
 
     def scan(self, i):
         if self.lib.vig_bigla_fwd_bf16(*self.calls[i % self.n_sets][1]) != 0:
@@ -303,8 +317,8 @@ def run_profile(args, cfg):
     torch.cuda.set_device(0)
     lib = vig.load()
     w = _Workload(cfg, lib, torch, torch.cuda.current_stream())
-    fn = {"fused": w.fused, "unfused": w.unfused, "scan": w.scan}[args.profile]
-    if args.profile == "scan":
+    fn = {"fused": w.fused, "unfused": w.unfused, "scan": w.scan, "bwd": w.bwd}[args.profile]
+    if args.profile in ("scan", "bwd"):
         w.unfused(0)   # log alpha of set 0 in place; the other sets' log alpha buffers hold arbitrary finite values
         for d in w.sets[1:]:
             d["la_f"].copy_(w.sets[0]["la_f"])
@@ -360,6 +374,7 @@ def run_gpu(args, cfg):
     unfused_ms, _, _ = w.time(w.unfused, args.steps, args.warmup, 20.0, dist, vdist)   # also leaves log alpha in place for the scan
     scan_ms, _, _ = w.time(w.scan, min(args.steps, 2000), args.warmup, 20.0, dist, vdist)
     blend_ms, _, _ = w.time(w.blend, min(args.steps, 2000), args.warmup, 20.0, dist, vdist)
+    bwd_ms, _, _ = w.time(w.bwd, min(args.steps, 200), args.warmup, 20.0, dist, vdist)
     assert vig.vig_last_device_status() == 0, "a device-side bounded wait expired"
     ms_per_step = float(np.median(step_ms))
     scan_us = float(np.median(scan_ms)) * 1e3
@@ -391,6 +406,17 @@ def run_gpu(args, cfg):
     blend_us = float(np.median(blend_ms)) * 1e3
     line["blend_step"] = dict(_summary(blend_ms), step="vig_bigla_fwd_blend_bf16", algorithmic_bytes=blend_bytes,
                               achieved_gbs=blend_bytes / (blend_us * 1e-6) / 1e9, frac=blend_bytes / (blend_us * 1e-6) / 1e9 / peak)
+
+    # the gradient call (log alpha and d_out in, five gradients out): 8 dk + 3 dv elements per token-head cross HBM; the two
+    # recurrence walks do 20 dk dv fp32 flops per token-head on the CUDA cores (peak: SMs x 128 lanes x 2 x max SM clock)
+    bwd_bytes = cfg.units * cfg.L * (8 * cfg.dk + 3 * cfg.dv) * cfg.elem_bytes
+    bwd_us = float(np.median(bwd_ms)) * 1e3
+    walk_flops = 20.0 * cfg.dk * cfg.dv * cfg.units * cfg.L
+    alu_peak = torch.cuda.get_device_properties(0).multi_processor_count * 128 * 2 * 1.965e9
+    line["bwd_step"] = dict(_summary(bwd_ms), step="vig_bigla_bwd_bf16", algorithmic_bytes=bwd_bytes,
+                            achieved_gbs=bwd_bytes / (bwd_us * 1e-6) / 1e9, frac_hbm=bwd_bytes / (bwd_us * 1e-6) / 1e9 / peak,
+                            walk_fp32_tflops=walk_flops / (bwd_us * 1e-6) / 1e12, frac_alu=walk_flops / (bwd_us * 1e-6) / alu_peak,
+                            tokens_per_s=tokens_per_step / (bwd_us * 1e-6))
 
     if rank == 0:
         # ---- end to end through the host-buffer entry point (H2D + kernels + D2H in the timed region) ----
@@ -467,7 +493,7 @@ def main():
     ap.add_argument("--only-headline", action="store_true", help="skip the shorter runs of the other bf16 workloads")
     ap.add_argument("--sweep", action="store_true",
                     help="also time the second workload (resolution sweep, hierarchical stage shapes) in the `workloads` object")
-    ap.add_argument("--profile", choices=["fused", "unfused", "scan"],
+    ap.add_argument("--profile", choices=["fused", "unfused", "scan", "bwd"],
                     help="for profilers: W warm-up and K steps of one call sequence only, nothing else is launched or timed")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

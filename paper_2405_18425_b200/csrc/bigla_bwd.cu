@@ -15,7 +15,7 @@
 // One block per unit walks the sequence twice.  The ascending walk carries S> and Z< and leaves dq>_t, dk<_t in fp32
 // scratch; the descending walk carries S< and Z>, reads them back and finishes all four outputs, the gate gradients as
 // running sums in walking order.  Thread (i, cg) keeps columns [cg CN, cg CN + CN) of row i of both dk x dv matrices in
-// registers; the sums over the value dimension are finished over the four lanes of a row by shuffles.  Inputs and
+// registers; the sums over the value dimension are finished over the two or four lanes of a row by shuffles.  Inputs and
 // outputs pass through shared memory sixteen tokens at a time, so global memory sees whole rows.
 #include <atomic>
 
@@ -27,128 +27,170 @@ namespace vig {
 namespace {
 
 constexpr int kBwdTT = 16;   // tokens staged at once
-constexpr int kBwdCG = 4;    // threads (lanes) per state row
 
 template <typename T>
 struct BwdArgs {
     const T *q, *k, *v, *la_f, *la_b, *g;
     T *dq, *dkey, *dla_f, *dla_b;
-    float* scratch;   // [units][2][L][dk] fp32: dq>, dk< between the two walks
+    float* scratch;   // [units][L][dk][2] fp32: (dq>, dk<) between the two walks
     long long units;
     int L, dk, dv;
 };
 
-// rows: state rows a block holds (threads / 4, >= dk); the padded rows and columns work on zeros.
-__host__ __device__ inline size_t bwd_smem_floats(int rows, int cn) {
-    return (size_t)kBwdTT * (10 * rows + 2 * kBwdCG * cn);
+// Two fp32 lanes per instruction (the packed fp32 arithmetic of sm_100: fma.rn.f32x2, mul.rn.f32x2; each lane rounds
+// like the scalar instruction).  A pair lives in one 64-bit register from the shared-memory load to the final sum, so
+// that no instruction is spent on packing.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+__device__ __forceinline__ float sum2(f32x2 a) {
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a));
+    return lo + hi;
+}
+__device__ __forceinline__ f32x2 ffma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 fmul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 
-template <typename T, int CN>
-__global__ void __launch_bounds__(512) bigla_bwd_kernel(BwdArgs<T> a) {
+// rows: state rows a block holds (threads / 4, >= dk); the padded rows and columns work on zeros.
+__host__ __device__ inline size_t bwd_smem_floats(int rows, int cn, int cg) {
+    return (size_t)kBwdTT * (10 * rows + 2 * cg * (cn + 4));   // (+ 4: a lane group's columns start 16 bytes off the
+                                                                   // bank of the group before it)
+}
+
+// CG: threads (adjacent lanes) per state row, 2 or 4.  CN: columns of the state per thread (a multiple of 4).  ROWS: state
+// rows of the block (threads / CG) when known at compile time - every shared-memory offset is then an immediate - or 0
+// for any block size.
+template <typename T, int CN, int ROWS, int CG>
+__global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdArgs<T> a) {
+    constexpr int kBwdCG = CG;
+    static_assert(CN % 4 == 0, "columns per thread come in 16-byte pieces");
     extern __shared__ __align__(16) float bw_smem[];
-    const int tid = threadIdx.x, nt = blockDim.x;
-    const int rows = nt / kBwdCG, cols = kBwdCG * CN;
+    const int tid = threadIdx.x, nt = ROWS ? ROWS * kBwdCG : blockDim.x;
+    const int rows = ROWS ? ROWS : nt / kBwdCG;
+    constexpr int cols = kBwdCG * (CN + 4);   // a token's row of v / d_out: CG groups of CN (+ 4 unused) floats
     const int i = tid / kBwdCG, cg = tid % kBwdCG;
     const int L = a.L, dk = a.dk, dv = a.dv;
-    float* qs = bw_smem;                      // [TT][rows] each
-    float* ks = qs + kBwdTT * rows;
-    float* a1 = ks + kBwdTT * rows;           // decay of the S state at this token
-    float* a2 = a1 + kBwdTT * rows;           // decay of the Z state: the gate of the token walked just before
-    float* x1 = a2 + kBwdTT * rows;           // descending walk: dq>, dk< from scratch
-    float* x2 = x1 + kBwdTT * rows;
-    float* o1 = x2 + kBwdTT * rows;           // results of sixteen tokens
-    float* o2 = o1 + kBwdTT * rows;
-    float* o3 = o2 + kBwdTT * rows;
-    float* o4 = o3 + kBwdTT * rows;
-    float* vs = o4 + kBwdTT * rows;           // [TT][cols] each
+    float4* rowd = reinterpret_cast<float4*>(bw_smem);                  // [TT][rows]: k, q, decay of S, decay of Z
+    float4* outd = rowd + kBwdTT * rows;                                // [TT][rows]: results of sixteen tokens
+    float2* xd = reinterpret_cast<float2*>(outd + kBwdTT * rows);       // [TT][rows]: dq>, dk< (descending walk)
+    float* vs = reinterpret_cast<float*>(xd + kBwdTT * rows);           // [TT][cols]
     float* gs = vs + kBwdTT * cols;
-    for (size_t x = tid; x < bwd_smem_floats(rows, CN); x += nt) bw_smem[x] = 0.f;   // the padding stays zero
+    for (size_t x = tid; x < bwd_smem_floats(rows, CN, CG); x += nt) bw_smem[x] = 0.f;   // the padding stays zero
     __syncthreads();
     const int nchunk = (L + kBwdTT - 1) / kBwdTT;
+    const int st_r = tid % rows, st_t = tid / rows;   // staging: thread = one key dimension of every fourth token
 
     for (long long unit = blockIdx.x; unit < a.units; unit += gridDim.x) {
         const size_t ok = (size_t)unit * L * dk, ov = (size_t)unit * L * dv;
-        float* sc1 = a.scratch + (size_t)unit * 2 * L * dk;
-        float* sc2 = sc1 + (size_t)L * dk;
+        float2* sc = reinterpret_cast<float2*>(a.scratch) + ok;   // [L][dk] pairs (dq>, dk<)
         for (int walk = 0; walk < 2; ++walk) {
-            const T* la_s = walk == 0 ? a.la_f : a.la_b;   // gates of the S state
-            const T* la_z = walk == 0 ? a.la_b : a.la_f;   // gates of the Z state
+            const T* la_s = (walk == 0 ? a.la_f : a.la_b) + ok;   // gates of the S state
+            const T* la_z = (walk == 0 ? a.la_b : a.la_f) + ok;   // gates of the Z state
             const int step = walk == 0 ? 1 : -1;
-            float S[CN], Z[CN];
+            f32x2 S[CN / 2], Z[CN / 2];
 #pragma unroll
-            for (int c = 0; c < CN; ++c) S[c] = Z[c] = 0.f;
+            for (int c = 0; c < CN / 2; ++c) S[c] = Z[c] = 0ull;   // (+0, +0)
             float run_f = 0.f, run_b = 0.f;   // running sums of E> and E< (descending walk)
             for (int cc = 0; cc < nchunk; ++cc) {
                 const int t0 = (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
                 const int nv = min(kBwdTT, L - t0);
-                for (int x = tid; x < nv * dk; x += nt) {
-                    const int tt = x / dk, r = x - tt * dk, t = t0 + tt;
-                    const size_t gi = ok + (size_t)t * dk + r;
-                    qs[tt * rows + r] = rec_to_float(a.q[gi]);
-                    ks[tt * rows + r] = rec_to_float(a.k[gi]);
-                    a1[tt * rows + r] = expf(rec_to_float(la_s[gi]));
-                    const int tp = t - step;   // the token walked before t
-                    a2[tt * rows + r] = (tp >= 0 && tp < L) ? expf(rec_to_float(la_z[ok + (size_t)tp * dk + r])) : 0.f;
-                    if (walk == 1) {
-                        x1[tt * rows + r] = sc1[(size_t)t * dk + r];
-                        x2[tt * rows + r] = sc2[(size_t)t * dk + r];
+                if (st_r < dk) {
+                    for (int tt = st_t; tt < nv; tt += kBwdCG) {
+                        const int t = t0 + tt, tp = t - step;   // tp: the token walked before t
+                        const size_t gi = (size_t)t * dk + st_r;
+                        float4 r4;
+                        r4.x = rec_to_float(a.k[ok + gi]);
+                        r4.y = rec_to_float(a.q[ok + gi]);
+                        r4.z = expf(rec_to_float(la_s[gi]));
+                        r4.w = (tp >= 0 && tp < L) ? expf(rec_to_float(la_z[(size_t)tp * dk + st_r])) : 0.f;
+                        rowd[tt * rows + st_r] = r4;
+                        if (walk == 1) xd[tt * rows + st_r] = sc[gi];
                     }
                 }
-                for (int x = tid; x < nv * dv; x += nt) {
-                    const int tt = x / dv, j = x - tt * dv;
-                    vs[tt * cols + j] = rec_to_float(a.v[ov + (size_t)(t0 + tt) * dv + j]);
-                    gs[tt * cols + j] = rec_to_float(a.g[ov + (size_t)(t0 + tt) * dv + j]);
+                {
+                    int tt = 0, j = tid;
+                    while (j >= dv) { j -= dv; ++tt; }
+                    while (tt < nv) {
+                        const int at = tt * cols + (j / CN) * (CN + 4) + j % CN;
+                        const size_t gi = ov + (size_t)(t0 + tt) * dv + j;
+                        vs[at] = rec_to_float(a.v[gi]);
+                        gs[at] = rec_to_float(a.g[gi]);
+                        j += nt;
+                        while (j >= dv) { j -= dv; ++tt; }
+                    }
                 }
                 __syncthreads();
-                for (int n = 0; n < nv; ++n) {
-                    const int tt = walk == 0 ? n : nv - 1 - n;
-                    const float kq = ks[tt * rows + i], qv = qs[tt * rows + i], hq = 0.5f * qv;
-                    const float ds = a1[tt * rows + i], dz = a2[tt * rows + i];
-                    const float* vr = vs + tt * cols + cg * CN;
-                    const float* gr = gs + tt * cols + cg * CN;
-                    float accq = 0.f, acck = 0.f;
+                {
+                    const float4* rp = rowd + (walk == 0 ? 0 : nv - 1) * rows + i;
+                    const float2* xp = xd + (walk == 0 ? 0 : nv - 1) * rows + i;
+                    float4* op = outd + (walk == 0 ? 0 : nv - 1) * rows + i;
+                    const float* vp = vs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
+                    const float* gp = gs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
+                    const int srow = step * rows, scol = step * cols;
+#pragma unroll 2
+                    for (int n = 0; n < nv; ++n, rp += srow, xp += srow, op += srow, vp += scol, gp += scol) {
+                        const float4 r4 = *rp;   // k, q, decay of S, decay of Z
+                        const float hq = 0.5f * r4.y;
+                        const ulonglong2* vr = reinterpret_cast<const ulonglong2*>(vp);   // two pairs each
+                        const ulonglong2* gr = reinterpret_cast<const ulonglong2*>(gp);
+                        const f32x2 ds2 = pack2(r4.z, r4.z), dz2 = pack2(r4.w, r4.w), kq2 = pack2(r4.x, r4.x), hq2 = pack2(hq, hq);
+                        f32x2 aq[2] = {0ull, 0ull}, ak[2] = {0ull, 0ull};
 #pragma unroll
-                    for (int c = 0; c < CN; ++c) {
-                        const float vj = vr[c], gj = gr[c];
-                        S[c] = fmaf(ds, S[c], kq * vj);
-                        accq = fmaf(S[c], gj, accq);
-                        Z[c] = fmaf(dz, Z[c], hq * gj);
-                        acck = fmaf(Z[c], vj, acck);
-                    }
-                    accq += __shfl_xor_sync(0xffffffffu, accq, 1);
-                    acck += __shfl_xor_sync(0xffffffffu, acck, 1);
-                    accq += __shfl_xor_sync(0xffffffffu, accq, 2);
-                    acck += __shfl_xor_sync(0xffffffffu, acck, 2);
-                    accq *= 0.5f;
-                    if (walk == 0) {
-                        if (cg == 0) {
-                            o1[tt * rows + i] = accq;   // dq>_t
-                            o2[tt * rows + i] = acck;   // dk<_t
+                        for (int c4 = 0; c4 < CN / 4; ++c4) {
+                            const ulonglong2 v4 = vr[c4], g4 = gr[c4];
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                const f32x2 vj = h == 0 ? v4.x : v4.y, gj = h == 0 ? g4.x : g4.y;
+                                const int c = 2 * c4 + h;
+                                S[c] = ffma2(ds2, S[c], fmul2(kq2, vj));   // S_t = a S + k^T v
+                                aq[h] = ffma2(S[c], gj, aq[h]);            // S_t g^T
+                                Z[c] = ffma2(dz2, Z[c], fmul2(hq2, gj));   // Z_t = a' Z + q^T g / 2
+                                ak[h] = ffma2(Z[c], vj, ak[h]);            // Z_t v^T
+                            }
                         }
-                    } else {
-                        const float dqf = x1[tt * rows + i], dkb = x2[tt * rows + i];   // accq = dq<_t, acck = dk>_t
-                        run_f += qv * dqf - kq * acck;
-                        if (cg == 0) {
-                            o1[tt * rows + i] = dqf + accq;
-                            o2[tt * rows + i] = acck + dkb;
-                            o3[tt * rows + i] = run_f;     // sum over m >= t of E>_m
-                            o4[tt * rows + i] = -run_b;    // minus the sum over m > t of E<_m
+                        float accq = sum2(aq[0]) + sum2(aq[1]), acck = sum2(ak[0]) + sum2(ak[1]);
+                        accq += __shfl_xor_sync(0xffffffffu, accq, 1);
+                        acck += __shfl_xor_sync(0xffffffffu, acck, 1);
+                        if (CG == 4) {
+                            accq += __shfl_xor_sync(0xffffffffu, accq, 2);
+                            acck += __shfl_xor_sync(0xffffffffu, acck, 2);
                         }
-                        run_b += qv * accq - kq * dkb;
+                        accq *= 0.5f;
+                        if (walk == 0) {
+                            if (cg == 0) *op = make_float4(accq, acck, 0.f, 0.f);   // dq>_t, dk<_t
+                        } else {
+                            const float2 x2 = *xp;   // dq>_t, dk<_t;  accq = dq<_t, acck = dk>_t
+                            run_f += r4.y * x2.x - r4.x * acck;
+                            // dq, dk, the sum over m >= t of E>_m, minus the sum over m > t of E<_m
+                            if (cg == 0) *op = make_float4(x2.x + accq, acck + x2.y, run_f, -run_b);
+                            run_b += r4.y * accq - r4.x * x2.y;
+                        }
                     }
                 }
                 __syncthreads();
-                for (int x = tid; x < nv * dk; x += nt) {
-                    const int tt = x / dk, r = x - tt * dk;
-                    const size_t t = (size_t)(t0 + tt);
-                    if (walk == 0) {
-                        sc1[t * dk + r] = o1[tt * rows + r];
-                        sc2[t * dk + r] = o2[tt * rows + r];
-                    } else {
-                        rec_store(a.dq + ok + t * dk + r, o1[tt * rows + r]);
-                        rec_store(a.dkey + ok + t * dk + r, o2[tt * rows + r]);
-                        rec_store(a.dla_f + ok + t * dk + r, o3[tt * rows + r]);
-                        rec_store(a.dla_b + ok + t * dk + r, o4[tt * rows + r]);
+                if (st_r < dk) {
+                    for (int tt = st_t; tt < nv; tt += kBwdCG) {
+                        const size_t gi = (size_t)(t0 + tt) * dk + st_r;
+                        const float4 o4 = outd[tt * rows + st_r];
+                        if (walk == 0) {
+                            sc[gi] = make_float2(o4.x, o4.y);
+                        } else {
+                            rec_store(a.dq + ok + gi, o4.x);
+                            rec_store(a.dkey + ok + gi, o4.y);
+                            rec_store(a.dla_f + ok + gi, o4.z);
+                            rec_store(a.dla_b + ok + gi, o4.w);
+                        }
                     }
                 }
                 // (the next chunk's staging writes other arrays; its results wait behind the barrier after staging)
@@ -175,30 +217,42 @@ __global__ void __launch_bounds__(256) shift_gates_kernel(const T* __restrict__ 
     }
 }
 
-template <typename T, int CN>
+template <typename T, int CN, int ROWS, int CG>
 cudaError_t launch_bwd_t(const BwdArgs<T>& a, int threads, int sms, cudaStream_t stream) {
-    const size_t smem = bwd_smem_floats(threads / kBwdCG, CN) * sizeof(float);
+    const size_t smem = bwd_smem_floats(threads / CG, CN, CG) * sizeof(float);
     static std::atomic<bool> configured[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev].load(std::memory_order_acquire)) {
-        if ((e = cudaFuncSetAttribute(bigla_bwd_kernel<T, CN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(bigla_bwd_kernel<T, CN, ROWS, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess)
+            return e;
         configured[dev].store(true, std::memory_order_release);
     }
     long long grid = a.units < 32LL * sms ? a.units : 32LL * sms;
-    bigla_bwd_kernel<T, CN><<<(unsigned)grid, threads, smem, stream>>>(a);
+    bigla_bwd_kernel<T, CN, ROWS, CG><<<(unsigned)grid, threads, smem, stream>>>(a);
     count_launch();
     return cudaGetLastError();
+}
+
+// Threads per key dimension.  Four: measured faster than two on the paper's shapes (768 units of 196 tokens: 411 us
+// against 524 us - fewer instructions with two, but too few warps to hide the latency of a step); two only where four
+// would leave a thread fewer than eight columns.
+int bwd_cg(int dv) { return dv >= 32 ? 4 : 2; }
+// ... in whole warps (the extra rows of the last warp work on zeros).
+int bwd_threads(int dk, int cg) { return (cg * dk + 31) / 32 * 32; }
+int bwd_cn(int dv, int cg) {   // columns per thread: the instantiated size that holds ceil(dv / cg)
+    const int cn = (dv + cg - 1) / cg;
+    return cn <= 8 ? 8 : (cn <= 12 ? 12 : (cn <= 16 ? 16 : (cn <= 24 ? 24 : 32)));
 }
 
 }  // namespace
 
 bool bwd_supported(int dk, int dv) {
     if (dk < 1 || dv < 1 || dk > 128 || dv > 128) return false;   // at most 512 threads, 32 columns per thread
-    const int threads = (kBwdCG * dk + 31) / 32 * 32, cn = (dv + kBwdCG - 1) / kBwdCG;
-    return bwd_smem_floats(threads / kBwdCG, cn <= 8 ? 8 : (cn <= 12 ? 12 : (cn <= 16 ? 16 : 32))) * sizeof(float) <= 200 * 1024;
+    const int cg = bwd_cg(dv), threads = bwd_threads(dk, cg);
+    return bwd_smem_floats(threads / cg, bwd_cn(dv, cg), cg) * sizeof(float) <= 200 * 1024;
 }
 
 size_t bwd_scratch_bytes(long long units, int L, int dk) { return (size_t)units * 2 * L * dk * sizeof(float); }
@@ -221,11 +275,18 @@ cudaError_t launch_bigla_bwd(const T* q, const T* k, const T* v, const T* la_f, 
     if (e != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     BwdArgs<T> a{q, k, v, la_f, la_b, d_out, dq, dk_out, dla_f, dla_b, scratch, units, L, dk, dv};
-    const int threads = (kBwdCG * dk + 31) / 32 * 32, cn = (dv + kBwdCG - 1) / kBwdCG;
-    if (cn <= 8) return launch_bwd_t<T, 8>(a, threads, sms, stream);
-    if (cn <= 12) return launch_bwd_t<T, 12>(a, threads, sms, stream);
-    if (cn <= 16) return launch_bwd_t<T, 16>(a, threads, sms, stream);
-    return launch_bwd_t<T, 32>(a, threads, sms, stream);
+    const int cg = bwd_cg(dv), threads = bwd_threads(dk, cg), cn = bwd_cn(dv, cg), rows = threads / cg;
+#define VIG_BWD_CASE(CN_, ROWS_, CG_) \
+    if (cn == CN_ && cg == CG_ && (ROWS_ == 0 || rows == ROWS_)) return launch_bwd_t<T, CN_, ROWS_, CG_>(a, threads, sms, stream);
+    if constexpr (sizeof(T) == 2) {   // the head sizes of the paper's models: block shape known at compile time
+        VIG_BWD_CASE(8, 16, 4) VIG_BWD_CASE(8, 24, 4) VIG_BWD_CASE(8, 32, 4)        // dv = 32; dk = 16, 24, 32
+        VIG_BWD_CASE(12, 16, 4) VIG_BWD_CASE(12, 24, 4) VIG_BWD_CASE(12, 32, 4)     // dv = 48
+        VIG_BWD_CASE(16, 16, 4) VIG_BWD_CASE(16, 24, 4) VIG_BWD_CASE(16, 32, 4)     // dv = 64
+    }
+    VIG_BWD_CASE(8, 0, 2) VIG_BWD_CASE(12, 0, 2) VIG_BWD_CASE(16, 0, 2)             // dv < 32
+    VIG_BWD_CASE(8, 0, 4) VIG_BWD_CASE(12, 0, 4) VIG_BWD_CASE(16, 0, 4) VIG_BWD_CASE(24, 0, 4) VIG_BWD_CASE(32, 0, 4)
+#undef VIG_BWD_CASE
+    return cudaErrorInvalidValue;
 }
 
 template cudaError_t launch_shift_gates<float>(const float*, const float*, float*, float*, long long, int, int, cudaStream_t);
