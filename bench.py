@@ -261,6 +261,21 @@ class _Workload:
         if self.lib.vig_bigla_fwd_blend_bf16(*self.calls[i % self.n_sets][3]) != 0:
             raise RuntimeError("vig_bigla_fwd_blend_bf16 failed")
 
+    def dwconv(self, i):
+        """Depth-wise 3x3 convolution of Eq. 7 over the patch grid of the configuration, [B, sqrt(L), sqrt(L), H dv] channels last:
+        the bytes of an O_local tensor serve as the image, those of `out` take the result."""
+        cfg, d = self.cfg, self.sets[i % self.n_sets]
+        side = int(round(cfg.L ** 0.5))
+        if side * side != cfg.L:
+            raise RuntimeError("the patch grid of this workload is not square")
+        if not hasattr(self, "dw_w"):
+            g = self.torch.Generator(device="cuda").manual_seed(cfg.seed)
+            self.dw_w = (self.torch.randn(cfg.H * cfg.dv, 3, 3, device="cuda", generator=g) / 3).to(self.torch.bfloat16)
+            self.dw_b = self.torch.randn(cfg.H * cfg.dv, device="cuda", generator=g).to(self.torch.bfloat16)
+        if self.lib.vig_dwconv3x3_bf16(d["o_local"].data_ptr(), self.dw_w.data_ptr(), self.dw_b.data_ptr(), d["out"].data_ptr(),
+                                       cfg.B, side, side, cfg.H * cfg.dv, self.stream.cuda_stream) != 0:
+            raise RuntimeError("vig_dwconv3x3_bf16 failed")
+
     def bwd(self, i):   # (log alpha of every set is in place once the un-fused step has run over the sets)
         if self.lib.vig_bigla_bwd_bf16(*self.calls[i % self.n_sets][4]) != 0:
             raise RuntimeError("vig_bigla_bwd_bf16 failed")
@@ -317,7 +332,7 @@ def run_profile(args, cfg):
     torch.cuda.set_device(0)
     lib = vig.load()
     w = _Workload(cfg, lib, torch, torch.cuda.current_stream())
-    fn = {"fused": w.fused, "unfused": w.unfused, "scan": w.scan, "bwd": w.bwd}[args.profile]
+    fn = {"fused": w.fused, "unfused": w.unfused, "scan": w.scan, "bwd": w.bwd, "dwconv": w.dwconv, "blend": w.blend}[args.profile]
     if args.profile in ("scan", "bwd"):
         w.unfused(0)   # log alpha of set 0 in place; the other sets' log alpha buffers hold arbitrary finite values
         for d in w.sets[1:]:
@@ -374,6 +389,7 @@ def run_gpu(args, cfg):
     unfused_ms, _, _ = w.time(w.unfused, args.steps, args.warmup, 20.0, dist, vdist)   # also leaves log alpha in place for the scan
     scan_ms, _, _ = w.time(w.scan, min(args.steps, 2000), args.warmup, 20.0, dist, vdist)
     blend_ms, _, _ = w.time(w.blend, min(args.steps, 2000), args.warmup, 20.0, dist, vdist)
+    dw_ms, _, _ = w.time(w.dwconv, min(args.steps, 2000), args.warmup, 10.0, dist, vdist)
     bwd_ms, _, _ = w.time(w.bwd, min(args.steps, 200), args.warmup, 20.0, dist, vdist)
     assert vig.vig_last_device_status() == 0, "a device-side bounded wait expired"
     ms_per_step = float(np.median(step_ms))
@@ -407,6 +423,11 @@ def run_gpu(args, cfg):
     line["blend_step"] = dict(_summary(blend_ms), step="vig_bigla_fwd_blend_bf16", algorithmic_bytes=blend_bytes,
                               achieved_gbs=blend_bytes / (blend_us * 1e-6) / 1e9, frac=blend_bytes / (blend_us * 1e-6) / 1e9 / peak)
 
+    # the depth-wise convolution in front of the mixer (Eq. 7 line 1): one read and one write of [B, L, H dv]
+    dw_bytes = 2 * cfg.units * cfg.L * cfg.dv * cfg.elem_bytes
+    dw_us = float(np.median(dw_ms)) * 1e3
+    line["dwconv_step"] = dict(_summary(dw_ms), step="vig_dwconv3x3_bf16", algorithmic_bytes=dw_bytes,
+                               achieved_gbs=dw_bytes / (dw_us * 1e-6) / 1e9, frac=dw_bytes / (dw_us * 1e-6) / 1e9 / peak)
     # the gradient call (log alpha and d_out in, five gradients out): 8 dk + 3 dv elements per token-head cross HBM; the two
     # recurrence walks do 20 dk dv fp32 flops per token-head on the CUDA cores (peak: SMs x 128 lanes x 2 x max SM clock)
     bwd_bytes = cfg.units * cfg.L * (8 * cfg.dk + 3 * cfg.dv) * cfg.elem_bytes
@@ -493,7 +514,7 @@ def main():
     ap.add_argument("--only-headline", action="store_true", help="skip the shorter runs of the other bf16 workloads")
     ap.add_argument("--sweep", action="store_true",
                     help="also time the second workload (resolution sweep, hierarchical stage shapes) in the `workloads` object")
-    ap.add_argument("--profile", choices=["fused", "unfused", "scan", "bwd"],
+    ap.add_argument("--profile", choices=["fused", "unfused", "scan", "bwd", "dwconv", "blend"],
                     help="for profilers: W warm-up and K steps of one call sequence only, nothing else is launched or timed")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

@@ -18,6 +18,7 @@
 // registers; the sums over the value dimension are finished over the two or four lanes of a row by shuffles.  Inputs and
 // outputs pass through shared memory sixteen tokens at a time, so global memory sees whole rows.
 #include <atomic>
+#include <cstring>
 
 #include "recurrence.cuh"
 #include "vig_internal.h"
@@ -204,16 +205,16 @@ __global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdAr
 // q, k swapped, the forward pass IS the gradient with respect to v:
 //   dv_r = 1/2 sum_{t >= r} (k_r * prod_{m = r+1..t} alpha>_m . q_t) g_t + 1/2 sum_{t <= r} (k_r * prod_{m = t..r-1} alpha<_m . q_t) g_t,
 // an anti-causal pass whose gate at "query" r .. "key" t - 1 is alpha>_{m+1}, and a causal one whose gate is alpha<_{m-1}.
-template <typename T>
-__global__ void __launch_bounds__(256) shift_gates_kernel(const T* __restrict__ la_f, const T* __restrict__ la_b, T* __restrict__ out_f,
-                                                          T* __restrict__ out_b, long long n, int L, int dk) {
+template <typename T, typename V>   // V: the unit moved per thread (T itself, or 16 bytes of T when a token's row is a whole number of them)
+__global__ void __launch_bounds__(256) shift_gates_kernel(const V* __restrict__ la_f, const V* __restrict__ la_b, V* __restrict__ out_f,
+                                                          V* __restrict__ out_b, long long n, int L, int row) {
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x; x < n; x += stride) {
-        const int t = (int)((x / dk) % L);
-        T zero;
-        rec_store(&zero, 0.f);
-        out_f[x] = t > 0 ? la_b[x - dk] : zero;
-        out_b[x] = t + 1 < L ? la_f[x + dk] : zero;
+        const int t = (int)((x / row) % L);
+        V zero;
+        memset(&zero, 0, sizeof(V));   // +0 in either type
+        out_f[x] = t > 0 ? la_b[x - row] : zero;
+        out_b[x] = t + 1 < L ? la_f[x + row] : zero;
     }
 }
 
@@ -259,10 +260,15 @@ size_t bwd_scratch_bytes(long long units, int L, int dk) { return (size_t)units 
 
 template <typename T>
 cudaError_t launch_shift_gates(const T* la_f, const T* la_b, T* out_f, T* out_b, long long units, int L, int dk, cudaStream_t stream) {
-    const long long n = units * L * dk;
+    const bool wide = (dk * sizeof(T)) % 16 == 0;   // (all four pointers are 16-byte aligned)
+    const int row = wide ? (int)(dk * sizeof(T) / 16) : dk;
+    const long long n = units * L * row;
     long long blocks = (n + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    shift_gates_kernel<T><<<(unsigned)blocks, 256, 0, stream>>>(la_f, la_b, out_f, out_b, n, L, dk);
+    if (wide)
+        shift_gates_kernel<T, uint4><<<(unsigned)blocks, 256, 0, stream>>>((const uint4*)la_f, (const uint4*)la_b, (uint4*)out_f, (uint4*)out_b, n, L, row);
+    else
+        shift_gates_kernel<T, T><<<(unsigned)blocks, 256, 0, stream>>>(la_f, la_b, out_f, out_b, n, L, row);
     count_launch();
     return cudaGetLastError();
 }
