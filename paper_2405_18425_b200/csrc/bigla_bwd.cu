@@ -16,7 +16,8 @@
 // scratch; the descending walk carries S< and Z>, reads them back and finishes all four outputs, the gate gradients as
 // running sums in walking order.  Thread (i, cg) keeps columns [cg CN, cg CN + CN) of row i of both dk x dv matrices in
 // registers; the sums over the value dimension are finished over the two or four lanes of a row by shuffles.  Inputs and
-// outputs pass through shared memory sixteen tokens at a time, so global memory sees whole rows.
+// outputs pass through shared memory sixteen tokens at a time: asynchronous copies (cp.async) bring the next sixteen
+// tokens in while the block works on these, where a token's row is a whole number of 16-byte pieces.
 #include <atomic>
 #include <cstring>
 
@@ -63,17 +64,29 @@ __device__ __forceinline__ f32x2 fmul2(f32x2 a, f32x2 b) {
     return d;
 }
 
-// rows: state rows a block holds (threads / 4, >= dk); the padded rows and columns work on zeros.
-__host__ __device__ inline size_t bwd_smem_floats(int rows, int cn, int cg) {
-    return (size_t)kBwdTT * (10 * rows + 2 * cg * (cn + 4));   // (+ 4: a lane group's columns start 16 bytes off the
-                                                                   // bank of the group before it)
+// Shared memory of a block.  rows: state rows it holds (threads / CG, >= dk; the padded rows and columns work on
+// zeros).  fp32 staging: 16-byte row records [TT][rows], the partial results read back [TT][rows] pairs, v and d_out
+// [TT][CG (cn + 4)] (+ 4: a lane group's columns start 16 bytes off the bank of the group before it); then the raw
+// landing zone of the asynchronous copies of the next sixteen tokens: k, q, two gate rows, v, d_out in the call's type
+// and the fp32 pairs.
+__host__ __device__ inline size_t bwd_stage_floats(int rows, int cn, int cg) { return (size_t)kBwdTT * (6 * rows + 2 * cg * (cn + 4)); }
+__host__ __device__ inline size_t bwd_smem_bytes(int rows, int cn, int cg, int dk, int dv, size_t elem) {
+    return bwd_stage_floats(rows, cn, cg) * sizeof(float) + (size_t)kBwdTT * ((4 * dk + 2 * dv) * elem + dk * 8) + 64;
 }
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+
+// Block shapes known at compile time are held to 85 registers (768 threads per SM: six blocks of 128).
+constexpr int bwd_max_threads(int rows, int cg) { return rows > 0 ? rows * cg : 512; }
+constexpr int bwd_min_blocks(int rows, int cg) { return rows > 0 ? 768 / (rows * cg) : 1; }
 
 // CG: threads (adjacent lanes) per state row, 2 or 4.  CN: columns of the state per thread (a multiple of 4).  ROWS: state
 // rows of the block (threads / CG) when known at compile time - every shared-memory offset is then an immediate - or 0
 // for any block size.
 template <typename T, int CN, int ROWS, int CG>
-__global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdArgs<T> a) {
+__global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS, CG)) bigla_bwd_kernel(BwdArgs<T> a) {
     constexpr int kBwdCG = CG;
     static_assert(CN % 4 == 0, "columns per thread come in 16-byte pieces");
     extern __shared__ __align__(16) float bw_smem[];
@@ -82,12 +95,21 @@ __global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdAr
     constexpr int cols = kBwdCG * (CN + 4);   // a token's row of v / d_out: CG groups of CN (+ 4 unused) floats
     const int i = tid / kBwdCG, cg = tid % kBwdCG;
     const int L = a.L, dk = a.dk, dv = a.dv;
-    float4* rowd = reinterpret_cast<float4*>(bw_smem);                  // [TT][rows]: k, q, decay of S, decay of Z
-    float4* outd = rowd + kBwdTT * rows;                                // [TT][rows]: results of sixteen tokens
-    float2* xd = reinterpret_cast<float2*>(outd + kBwdTT * rows);       // [TT][rows]: dq>, dk< (descending walk)
+    float4* rowd = reinterpret_cast<float4*>(bw_smem);                  // [TT][rows]: k, q, decay of S, decay of Z; then the results
+    float2* xd = reinterpret_cast<float2*>(rowd + kBwdTT * rows);       // [TT][rows]: dq>, dk< (descending walk)
     float* vs = reinterpret_cast<float*>(xd + kBwdTT * rows);           // [TT][cols]
     float* gs = vs + kBwdTT * cols;
-    for (size_t x = tid; x < bwd_smem_floats(rows, CN, CG); x += nt) bw_smem[x] = 0.f;   // the padding stays zero
+    // raw landing zone (16-byte aligned pieces): k, q, gates of S, gates of Z, v, d_out as stored, then the fp32 pairs
+    T* raw_k = reinterpret_cast<T*>(gs + kBwdTT * cols);
+    T* raw_q = raw_k + kBwdTT * dk;
+    T* raw_s = raw_q + kBwdTT * dk;
+    T* raw_z = raw_s + kBwdTT * dk;
+    T* raw_v = raw_z + kBwdTT * dk;
+    T* raw_g = raw_v + kBwdTT * dv;
+    float2* raw_x = reinterpret_cast<float2*>(raw_g + kBwdTT * dv);
+    // Rows of whole 16-byte pieces: the next sixteen tokens are copied asynchronously while these are worked on.
+    const bool ahead = (dk * sizeof(T)) % 16 == 0 && (dv * sizeof(T)) % 16 == 0;
+    for (size_t x = tid; x < bwd_stage_floats(rows, CN, CG); x += nt) bw_smem[x] = 0.f;   // the padding stays zero
     __syncthreads();
     const int nchunk = (L + kBwdTT - 1) / kBwdTT;
     const int st_r = tid % rows, st_t = tid / rows;   // staging: thread = one key dimension of every fourth token
@@ -103,39 +125,81 @@ __global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdAr
 #pragma unroll
             for (int c = 0; c < CN / 2; ++c) S[c] = Z[c] = 0ull;   // (+0, +0)
             float run_f = 0.f, run_b = 0.f;   // running sums of E> and E< (descending walk)
+            // sixteen tokens of every input on their way into the landing zone (thread = 16-byte pieces)
+            auto fetch = [&](int cc) {
+                const int t0 = (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
+                const int nv = min(kBwdTT, L - t0);
+                const int pk = nv * dk * (int)sizeof(T) / 16, pv = nv * dv * (int)sizeof(T) / 16, row16 = dk * (int)sizeof(T) / 16;
+                const char* gk = reinterpret_cast<const char*>(a.k + ok + (size_t)t0 * dk);
+                const char* gq = reinterpret_cast<const char*>(a.q + ok + (size_t)t0 * dk);
+                const char* gs_ = reinterpret_cast<const char*>(la_s + (size_t)t0 * dk);
+                for (int x = tid; x < pk; x += nt) {
+                    cp_async16(reinterpret_cast<char*>(raw_k) + 16 * x, gk + 16 * x);
+                    cp_async16(reinterpret_cast<char*>(raw_q) + 16 * x, gq + 16 * x);
+                    cp_async16(reinterpret_cast<char*>(raw_s) + 16 * x, gs_ + 16 * x);
+                    const int tp = t0 + x / row16 - step;   // slot tt of the Z gates holds token t0 + tt - step, where it exists
+                    if (tp >= 0 && tp < L)
+                        cp_async16(reinterpret_cast<char*>(raw_z) + 16 * x, reinterpret_cast<const char*>(la_z + (size_t)tp * dk) + 16 * (x % row16));
+                }
+                const char* gv = reinterpret_cast<const char*>(a.v + ov + (size_t)t0 * dv);
+                const char* gg = reinterpret_cast<const char*>(a.g + ov + (size_t)t0 * dv);
+                for (int x = tid; x < pv; x += nt) {
+                    cp_async16(reinterpret_cast<char*>(raw_v) + 16 * x, gv + 16 * x);
+                    cp_async16(reinterpret_cast<char*>(raw_g) + 16 * x, gg + 16 * x);
+                }
+                if (walk == 1) {
+                    const char* gx = reinterpret_cast<const char*>(sc + (size_t)t0 * dk);
+                    for (int x = tid; x < nv * dk / 2; x += nt) cp_async16(reinterpret_cast<char*>(raw_x) + 16 * x, gx + 16 * x);
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+            // sixteen tokens from `k_` ... (the landing zone, or global memory itself) into the fp32 staging
+            auto convert = [&](const T* k_, const T* q_, const T* s_, const T* z_, const T* v_, const T* g_, const float2* x_, int t0, int nv) {
+                if (st_r < dk) {
+                    for (int tt = st_t; tt < nv; tt += kBwdCG) {
+                        const int tp = t0 + tt - step;   // the token walked before this one
+                        const int e = tt * dk + st_r;
+                        float4 r4;
+                        r4.x = rec_to_float(k_[e]);
+                        r4.y = rec_to_float(q_[e]);
+                        r4.z = expf(rec_to_float(s_[e]));
+                        r4.w = (tp >= 0 && tp < L) ? expf(rec_to_float(z_[e])) : 0.f;
+                        rowd[tt * rows + st_r] = r4;
+                        if (walk == 1) xd[tt * rows + st_r] = x_[e];
+                    }
+                }
+                int tt = 0, j = tid;
+                while (j >= dv) { j -= dv; ++tt; }
+                while (tt < nv) {
+                    const int at = tt * cols + (j / CN) * (CN + 4) + j % CN;
+                    vs[at] = rec_to_float(v_[tt * dv + j]);
+                    gs[at] = rec_to_float(g_[tt * dv + j]);
+                    j += nt;
+                    while (j >= dv) { j -= dv; ++tt; }
+                }
+            };
+            if (ahead) fetch(0);
             for (int cc = 0; cc < nchunk; ++cc) {
                 const int t0 = (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
                 const int nv = min(kBwdTT, L - t0);
-                if (st_r < dk) {
-                    for (int tt = st_t; tt < nv; tt += kBwdCG) {
-                        const int t = t0 + tt, tp = t - step;   // tp: the token walked before t
-                        const size_t gi = (size_t)t * dk + st_r;
-                        float4 r4;
-                        r4.x = rec_to_float(a.k[ok + gi]);
-                        r4.y = rec_to_float(a.q[ok + gi]);
-                        r4.z = expf(rec_to_float(la_s[gi]));
-                        r4.w = (tp >= 0 && tp < L) ? expf(rec_to_float(la_z[(size_t)tp * dk + st_r])) : 0.f;
-                        rowd[tt * rows + st_r] = r4;
-                        if (walk == 1) xd[tt * rows + st_r] = sc[gi];
-                    }
+                if (ahead) {
+                    asm volatile("cp.async.wait_group 0;" ::: "memory");
+                    __syncthreads();   // everybody's pieces have landed (and the results of the chunk before are stored)
+                    convert(raw_k, raw_q, raw_s, raw_z, raw_v, raw_g, raw_x, t0, nv);
+                    __syncthreads();
+                    if (cc + 1 < nchunk) fetch(cc + 1);
+                } else {
+                    __syncthreads();   // the results of the chunk before are stored
+                    // (slot tt of the Z gates: token t0 + tt - step; the pointer is only followed where that token exists)
+                    convert(a.k + ok + (size_t)t0 * dk, a.q + ok + (size_t)t0 * dk, la_s + (size_t)t0 * dk,
+                            la_z + ((ptrdiff_t)t0 - step) * dk, a.v + ov + (size_t)t0 * dv, a.g + ov + (size_t)t0 * dv, sc + (size_t)t0 * dk, t0, nv);
+                    __syncthreads();
                 }
-                {
-                    int tt = 0, j = tid;
-                    while (j >= dv) { j -= dv; ++tt; }
-                    while (tt < nv) {
-                        const int at = tt * cols + (j / CN) * (CN + 4) + j % CN;
-                        const size_t gi = ov + (size_t)(t0 + tt) * dv + j;
-                        vs[at] = rec_to_float(a.v[gi]);
-                        gs[at] = rec_to_float(a.g[gi]);
-                        j += nt;
-                        while (j >= dv) { j -= dv; ++tt; }
-                    }
-                }
-                __syncthreads();
                 {
                     const float4* rp = rowd + (walk == 0 ? 0 : nv - 1) * rows + i;
                     const float2* xp = xd + (walk == 0 ? 0 : nv - 1) * rows + i;
-                    float4* op = outd + (walk == 0 ? 0 : nv - 1) * rows + i;
+                    float4* op = rowd + (walk == 0 ? 0 : nv - 1) * rows + i;   // the record is replaced by the results (the lanes of a
+                                                                                // row read it in the same instruction, before this lane writes)
                     const float* vp = vs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
                     const float* gp = gs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
                     const int srow = step * rows, scol = step * cols;
@@ -183,7 +247,7 @@ __global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdAr
                 if (st_r < dk) {
                     for (int tt = st_t; tt < nv; tt += kBwdCG) {
                         const size_t gi = (size_t)(t0 + tt) * dk + st_r;
-                        const float4 o4 = outd[tt * rows + st_r];
+                        const float4 o4 = rowd[tt * rows + st_r];
                         if (walk == 0) {
                             sc[gi] = make_float2(o4.x, o4.y);
                         } else {
@@ -194,7 +258,6 @@ __global__ void __launch_bounds__(ROWS ? ROWS * CG : 512) bigla_bwd_kernel(BwdAr
                         }
                     }
                 }
-                // (the next chunk's staging writes other arrays; its results wait behind the barrier after staging)
             }
             __syncthreads();   // the scratch of the ascending walk is read back by other threads
         }
@@ -220,7 +283,7 @@ __global__ void __launch_bounds__(256) shift_gates_kernel(const V* __restrict__ 
 
 template <typename T, int CN, int ROWS, int CG>
 cudaError_t launch_bwd_t(const BwdArgs<T>& a, int threads, int sms, cudaStream_t stream) {
-    const size_t smem = bwd_smem_floats(threads / CG, CN, CG) * sizeof(float);
+    const size_t smem = bwd_smem_bytes(threads / CG, CN, CG, a.dk, a.dv, sizeof(T));
     static std::atomic<bool> configured[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -253,7 +316,7 @@ int bwd_cn(int dv, int cg) {   // columns per thread: the instantiated size that
 bool bwd_supported(int dk, int dv) {
     if (dk < 1 || dv < 1 || dk > 128 || dv > 128) return false;   // at most 512 threads, 32 columns per thread
     const int cg = bwd_cg(dv), threads = bwd_threads(dk, cg);
-    return bwd_smem_floats(threads / cg, bwd_cn(dv, cg), cg) * sizeof(float) <= 200 * 1024;
+    return bwd_smem_bytes(threads / cg, bwd_cn(dv, cg), cg, dk, dv, 4) <= 200 * 1024;
 }
 
 size_t bwd_scratch_bytes(long long units, int L, int dk) { return (size_t)units * 2 * L * dk * sizeof(float); }
