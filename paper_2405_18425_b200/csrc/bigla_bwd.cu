@@ -74,6 +74,22 @@ __host__ __device__ inline size_t bwd_smem_bytes(int rows, int cn, int cg, int d
     return bwd_stage_floats(rows, cn, cg) * sizeof(float) + (size_t)kBwdTT * ((4 * dk + 2 * dv) * elem + dk * 8) + 64;
 }
 
+// Four consecutive elements of the call's type <-> fp32
+__device__ __forceinline__ void load4(const float* p, float (&f)[4]) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&f)[4]) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+__device__ __forceinline__ void store4(float* p, const float (&f)[4]) { *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]); }
+__device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&f)[4]) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(f[0], f[1]), hi = __floats2bfloat162_rn(f[2], f[3]);
+    *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+}
+
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
 }
@@ -178,6 +194,36 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                     while (j >= dv) { j -= dv; ++tt; }
                 }
             };
+            // the same from the landing zone, four elements at a time (rows are whole 16-byte pieces there)
+            auto convert4 = [&](int t0, int nv) {
+                const int qk = dk / 4, qv = dv / 4;
+                for (int x = tid; x < nv * qk; x += nt) {
+                    const int tt = x / qk, r0 = (x - tt * qk) * 4, e = tt * dk + r0, tp = t0 + tt - step;
+                    float kf[4], qf[4], sf[4], zf[4];
+                    load4(raw_k + e, kf);
+                    load4(raw_q + e, qf);
+                    load4(raw_s + e, sf);
+                    load4(raw_z + e, zf);
+                    const bool zin = tp >= 0 && tp < L;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) rowd[tt * rows + r0 + u] = make_float4(kf[u], qf[u], expf(sf[u]), zin ? expf(zf[u]) : 0.f);
+                    if (walk == 1) {
+                        const float4 xa = *reinterpret_cast<const float4*>(raw_x + e), xb = *reinterpret_cast<const float4*>(raw_x + e + 2);
+                        float4* xo = reinterpret_cast<float4*>(xd + tt * rows + r0);
+                        xo[0] = xa;
+                        xo[1] = xb;
+                    }
+                }
+                for (int x = tid; x < nv * qv; x += nt) {
+                    const int tt = x / qv, j0 = (x - tt * qv) * 4;
+                    const int at = tt * cols + (j0 / CN) * (CN + 4) + j0 % CN;
+                    float f[4];
+                    load4(raw_v + tt * dv + j0, f);
+                    store4(vs + at, f);
+                    load4(raw_g + tt * dv + j0, f);
+                    store4(gs + at, f);
+                }
+            };
             if (ahead) fetch(0);
             for (int cc = 0; cc < nchunk; ++cc) {
                 const int t0 = (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
@@ -185,7 +231,7 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                 if (ahead) {
                     asm volatile("cp.async.wait_group 0;" ::: "memory");
                     __syncthreads();   // everybody's pieces have landed (and the results of the chunk before are stored)
-                    convert(raw_k, raw_q, raw_s, raw_z, raw_v, raw_g, raw_x, t0, nv);
+                    convert4(t0, nv);
                     __syncthreads();
                     if (cc + 1 < nchunk) fetch(cc + 1);
                 } else {
@@ -244,7 +290,29 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                     }
                 }
                 __syncthreads();
-                if (st_r < dk) {
+                if (ahead) {   // four key dimensions of a token per thread: 8- or 16-byte stores
+                    const int qk = dk / 4;
+                    for (int x = tid; x < nv * qk; x += nt) {
+                        const int tt = x / qk, r0 = (x - tt * qk) * 4;
+                        const size_t gi = (size_t)(t0 + tt) * dk + r0;
+                        float o[4][4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const float4 o4 = rowd[tt * rows + r0 + u];
+                            o[0][u] = o4.x; o[1][u] = o4.y; o[2][u] = o4.z; o[3][u] = o4.w;
+                        }
+                        if (walk == 0) {
+                            float4* so = reinterpret_cast<float4*>(sc + gi);
+                            so[0] = make_float4(o[0][0], o[1][0], o[0][1], o[1][1]);
+                            so[1] = make_float4(o[0][2], o[1][2], o[0][3], o[1][3]);
+                        } else {
+                            store4(a.dq + ok + gi, o[0]);
+                            store4(a.dkey + ok + gi, o[1]);
+                            store4(a.dla_f + ok + gi, o[2]);
+                            store4(a.dla_b + ok + gi, o[3]);
+                        }
+                    }
+                } else if (st_r < dk) {
                     for (int tt = st_t; tt < nv; tt += kBwdCG) {
                         const size_t gi = (size_t)(t0 + tt) * dk + st_r;
                         const float4 o4 = rowd[tt * rows + st_r];
