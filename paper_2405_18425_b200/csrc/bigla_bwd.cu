@@ -90,6 +90,12 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&f)[4]) {
     *reinterpret_cast<uint2*>(p) = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
 }
 
+// 16-byte store to shared memory that the compiler does not take for a store to the C++ objects it tracks: the loads of
+// the tokens after this one may move above it (they never read what it writes; whoever reads it does so behind a barrier).
+__device__ __forceinline__ void sts128_untracked(void* p, float x, float y, float z, float w) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "f"(x), "f"(y), "f"(z), "f"(w));
+}
+
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
 }
@@ -249,7 +255,7 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                     const float* vp = vs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
                     const float* gp = gs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
                     const int srow = step * rows, scol = step * cols;
-#pragma unroll 2
+#pragma unroll 4
                     for (int n = 0; n < nv; ++n, rp += srow, xp += srow, op += srow, vp += scol, gp += scol) {
                         const float4 r4 = *rp;   // k, q, decay of S, decay of Z
                         const float hq = 0.5f * r4.y;
@@ -279,12 +285,12 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         }
                         accq *= 0.5f;
                         if (walk == 0) {
-                            if (cg == 0) *op = make_float4(accq, acck, 0.f, 0.f);   // dq>_t, dk<_t
+                            if (cg == 0) sts128_untracked(op, accq, acck, 0.f, 0.f);   // dq>_t, dk<_t
                         } else {
                             const float2 x2 = *xp;   // dq>_t, dk<_t;  accq = dq<_t, acck = dk>_t
                             run_f += r4.y * x2.x - r4.x * acck;
                             // dq, dk, the sum over m >= t of E>_m, minus the sum over m > t of E<_m
-                            if (cg == 0) *op = make_float4(x2.x + accq, acck + x2.y, run_f, -run_b);
+                            if (cg == 0) sts128_untracked(op, x2.x + accq, acck + x2.y, run_f, -run_b);
                             run_b += r4.y * accq - r4.x * x2.y;
                         }
                     }
