@@ -21,6 +21,7 @@
 #include <atomic>
 #include <cstring>
 
+#include "ptx.cuh"
 #include "recurrence.cuh"
 #include "vig_internal.h"
 
@@ -38,31 +39,6 @@ struct BwdArgs {
     long long units;
     int L, dk, dv;
 };
-
-// Two fp32 lanes per instruction (the packed fp32 arithmetic of sm_100: fma.rn.f32x2, mul.rn.f32x2; each lane rounds
-// like the scalar instruction).  A pair lives in one 64-bit register from the shared-memory load to the final sum, so
-// that no instruction is spent on packing.
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
-    f32x2 d;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
-    return d;
-}
-__device__ __forceinline__ float sum2(f32x2 a) {
-    float lo, hi;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(a));
-    return lo + hi;
-}
-__device__ __forceinline__ f32x2 ffma2(f32x2 a, f32x2 b, f32x2 c) {
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ f32x2 fmul2(f32x2 a, f32x2 b) {
-    f32x2 d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 
 // Shared memory of a block.  rows: state rows it holds (threads / CG, >= dk; the padded rows and columns work on
 // zeros).  fp32 staging: 16-byte row records [TT][rows], the partial results read back [TT][rows] pairs, v and d_out

@@ -20,6 +20,7 @@ struct Vec<float> {
     using Raw = float4;
     static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&f)[4]) { f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w; }
+    static __device__ __forceinline__ void unpack2x(const Raw& v, f32x2 (&f)[2]) { f[0] = pack2(v.x, v.y); f[1] = pack2(v.z, v.w); }
     static __device__ __forceinline__ void load(const float* p, float (&f)[4]) { unpack(*reinterpret_cast<const float4*>(p), f); }
     static __device__ __forceinline__ void store(float* p, const float (&f)[4]) {
         *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
@@ -39,6 +40,11 @@ struct Vec<__nv_bfloat16> {
             f[2 * x + 1] = t.y;
         }
     }
+    static __device__ __forceinline__ void unpack2x(const Raw& v, f32x2 (&f)[4]) {   // a bf16 is the upper half of its fp32
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int x = 0; x < 4; ++x) f[x] = pack2(__uint_as_float(w[x] << 16), __uint_as_float(w[x] & 0xffff0000u));
+    }
     static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) { unpack(*reinterpret_cast<const uint4*>(p), f); }
     static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&f)[8]) {
         *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
@@ -56,7 +62,7 @@ __device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float
 // input element crosses L2 once per tile that needs it instead of nine times.  A block keeps its slab (blockIdx.y) and
 // strides over tasks with two tile buffers: the next tile loads while this one is worked on.
 // Thread = one channel group of one column: its V filters (nine taps each, 144 contiguous bytes of w) and biases sit
-// in registers as fp32; walking down the tile it reads three 16-byte pieces per input row (left, centre, right) from
+// in registers as fp32 pairs (two channels per packed multiply-add); walking down the tile it reads three 16-byte pieces per input row (left, centre, right) from
 // shared memory and adds them into the three output rows they touch, which live in rolling accumulators.  Lanes run
 // over channel groups first, so shared-memory reads and the 16-byte output stores are contiguous per warp.
 template <typename T>
@@ -87,9 +93,9 @@ __global__ void __launch_bounds__(256) dwconv3x3_kernel(const __grid_constant__ 
     };
     pdl_wait();   // x may be the output of the kernel before this one in the stream
     if (threadIdx.x == 0 && (int)blockIdx.x < tasks) issue(blockIdx.x, 0);
-    float wr[9][V], br[V];
+    f32x2 wr[9][V / 2], br[V / 2];   // filter taps and biases of the thread's channels as fp32 pairs
 #pragma unroll
-    for (int u = 0; u < V; ++u) br[u] = 0.f;
+    for (int u = 0; u < V / 2; ++u) br[u] = 0ull;
     if (chan_live) {
         float t[9 * V];   // w[c0 .. c0 + V)[3][3]: 9 V contiguous elements = nine 16-byte pieces
 #pragma unroll
@@ -102,8 +108,13 @@ __global__ void __launch_bounds__(256) dwconv3x3_kernel(const __grid_constant__ 
 #pragma unroll
         for (int tap = 0; tap < 9; ++tap)
 #pragma unroll
-            for (int u = 0; u < V; ++u) wr[tap][u] = t[u * 9 + tap];
-        if (bias) Vec<T>::load(bias + c0, br);
+            for (int u = 0; u < V / 2; ++u) wr[tap][u] = pack2(t[(2 * u) * 9 + tap], t[(2 * u + 1) * 9 + tap]);
+        if (bias) {
+            float f[V];
+            Vec<T>::load(bias + c0, f);
+#pragma unroll
+            for (int u = 0; u < V / 2; ++u) br[u] = pack2(f[2 * u], f[2 * u + 1]);
+        }
     }
     const uint32_t row_pitch_s = (uint32_t)(tw + 2) * gpb * 16;   // one tile row in shared memory
     const size_t row_pitch_g = (size_t)Ww * C;
@@ -123,28 +134,33 @@ __global__ void __launch_bounds__(256) dwconv3x3_kernel(const __grid_constant__ 
             const uint8_t* tp = dw_smem + buf * buf_pitch + ((uint32_t)col * gpb + g) * 16;   // tile row 0, column j - 1
             T* op = out + (((size_t)n * Hh + i0) * Ww + j) * C + c0;
             // a_up: the output row above the input row at hand (complete with it), a_mid: the one at it, a_dn: the one below
-            float a_up[V], a_mid[V];
+            f32x2 a_up[V / 2], a_mid[V / 2];
 #pragma unroll
-            for (int u = 0; u < V; ++u) a_up[u] = a_mid[u] = br[u];
+            for (int u = 0; u < V / 2; ++u) a_up[u] = a_mid[u] = br[u];
             for (int r = 0; r < rows + 2; ++r) {   // tile row r = input row i0 - 1 + r (zeros outside the image)
-                float in[3][V];
+                f32x2 in[3][V / 2];
 #pragma unroll
                 for (int d = 0; d < 3; ++d)
-                    Vec<T>::unpack(*reinterpret_cast<const Raw*>(tp + (uint32_t)r * row_pitch_s + (uint32_t)d * gpb * 16), in[d]);
-                float a_dn[V];
+                    Vec<T>::unpack2x(*reinterpret_cast<const Raw*>(tp + (uint32_t)r * row_pitch_s + (uint32_t)d * gpb * 16), in[d]);
+                f32x2 a_dn[V / 2];
 #pragma unroll
-                for (int u = 0; u < V; ++u) {
+                for (int u = 0; u < V / 2; ++u) {   // two channels per instruction (packed fp32 multiply-add)
                     a_dn[u] = br[u];
 #pragma unroll
                     for (int d = 0; d < 3; ++d) {
-                        a_up[u] = fmaf(wr[6 + d][u], in[d][u], a_up[u]);
-                        a_mid[u] = fmaf(wr[3 + d][u], in[d][u], a_mid[u]);
-                        a_dn[u] = fmaf(wr[d][u], in[d][u], a_dn[u]);
+                        a_up[u] = ffma2(wr[6 + d][u], in[d][u], a_up[u]);
+                        a_mid[u] = ffma2(wr[3 + d][u], in[d][u], a_mid[u]);
+                        a_dn[u] = ffma2(wr[d][u], in[d][u], a_dn[u]);
                     }
                 }
-                if (r >= 2) Vec<T>::store(op + (size_t)(r - 2) * row_pitch_g, a_up);
+                if (r >= 2) {
+                    float o[V];
 #pragma unroll
-                for (int u = 0; u < V; ++u) {
+                    for (int u = 0; u < V / 2; ++u) unpack2(a_up[u], o[2 * u], o[2 * u + 1]);
+                    Vec<T>::store(op + (size_t)(r - 2) * row_pitch_g, o);
+                }
+#pragma unroll
+                for (int u = 0; u < V / 2; ++u) {
                     a_up[u] = a_mid[u];
                     a_mid[u] = a_dn[u];
                 }
