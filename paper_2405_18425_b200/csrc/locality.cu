@@ -226,7 +226,8 @@ cudaError_t launch_dwconv3x3(const T* x, const T* w, const T* bias, T* out, long
     constexpr int V = (int)(16 / sizeof(T));
     const int groups = C / V;
     const int slabs = (groups + 15) / 16, gpb = (groups + slabs - 1) / slabs;   // channel groups per block: at most 16
-    const int coltiles = (Ww + 256 / gpb - 1) / (256 / gpb), tw = (Ww + coltiles - 1) / coltiles;   // at most 256 threads, 256 columns
+    const int tw_max = 256 / gpb < 254 ? 256 / gpb : 254;   // at most 256 threads; the tile with its halo at most 256 columns (a TMA box)
+    const int coltiles = (Ww + tw_max - 1) / tw_max, tw = (Ww + coltiles - 1) / coltiles;
     const int rowsegs = (Hh + 7) / 8, th = (Hh + rowsegs - 1) / rowsegs;                            // at most 8 output rows per tile
     const long long tasks = images * rowsegs * coltiles;
     if (tasks > 0x7fffffffLL || slabs > 65535 || tw + 2 > 256) return cudaErrorInvalidValue;

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("B,Hh,Ww,C", [(2, 14, 14, 192), (1, 1, 1, 8), (3, 1, 9, 16), (2, 7, 1, 24), (1, 56, 56, 96),
-                                       (2, 5, 6, 1024), (1, 64, 64, 200)])
+                                       (2, 5, 6, 1024), (1, 64, 64, 200), (1, 3, 300, 8), (1, 19, 257, 8)])
 def test_dwconv3x3_matches_oracle(oracle, dtype, B, Hh, Ww, C):
     """Grids with a single row, a single column or a single pixel (only some taps exist), the patch grids of the
     configurations, channel counts that are not powers of two; bias given and absent."""
