@@ -417,7 +417,7 @@ def run_gpu(args, cfg):
         "clocks": clocks, "gpu_launches": int(launches),
     }
     line["roofline_step"]["traffic"] = None   # no capture of the fused kernel yet
-    # the layer's call with the 2-D gate blend of the locality injection in the epilogue: two more [B,H,L,dv] inputs
+    # the layer's call with the 2-D gate blend of the locality injection behind the forward pass: two more [B,H,L,dv] inputs
     blend_bytes = cfg.algorithmic_bytes + 2 * cfg.units * cfg.L * cfg.dv * cfg.elem_bytes
     blend_us = float(np.median(blend_ms)) * 1e3
     line["blend_step"] = dict(_summary(blend_ms), step="vig_bigla_fwd_blend_bf16", algorithmic_bytes=blend_bytes,

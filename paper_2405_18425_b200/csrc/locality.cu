@@ -1,7 +1,8 @@
 // The two element-wise neighbours of BiGLA in the 2-D gating locality injection (paper Eq. 7):
 //   line 1     O_local = DWConv3x3(X): depth-wise 3 x 3 convolution over the patch grid (channels last)
 //   lines 3-4  O = G * O_local + (1 - G) * O_global with G = sigmoid(z), z = O_local W + b given by the caller
-// Both are bound by memory traffic; the blend also exists as the epilogue of the forward kernel (bigla_umma.cu).
+// The blend is bound by memory traffic; the convolution reads every input once through tiled TMA loads and is then
+// bound by its multiply-adds.
 #include <atomic>
 
 #include "ptx.cuh"

@@ -1,5 +1,5 @@
 """GPU parity of the 2-D gating locality injection around the mixer (paper Eq. 7): the depth-wise 3x3 convolution, the
-gate blend on its own, and the blend fused into the forward pass, each against the fp64 oracle (oracle/locality.py and
+gate blend on its own, and the blend in the same call as the forward pass, each against the fp64 oracle (oracle/locality.py and
 the Eq. 6 recurrence) on the same seeded inputs.  Bars as for the mixer: 1e-4 (fp32) / 2e-2 (bf16) of max|oracle|."""
 import numpy as np
 import pytest
