@@ -68,6 +68,19 @@ def test_gradient_strong_gates(oracle):
     _check(got, ref, "f32")
 
 
+def test_bf16_gradient_with_a_unit_beyond_the_tensor_core_range(oracle):
+    """One unit whose gates sum to about -80 over a chunk: the forward kernel that supplies dv hands that unit to its
+    in-kernel recurrence (the counter says so); all five gradients must still meet the bar."""
+    cfg, x = random_problem(4300, 2, 3, 196, 32, 64, "bf16", gate_mean=1.0)
+    g = synth.stored_to_f64(x["g_bwd"], "bf16").copy()
+    g[1, 1, 10:140] = -10.0            # log alpha< = -10 / 16 per token; moved by one token it gates dv's forward pass
+    x["g_bwd"] = synth.store(g, "bf16")
+    vig.vig_test_take_fallback_count()
+    got, ref = _run(oracle, cfg, x, synth.make_grad_input(cfg))
+    assert vig.vig_test_take_fallback_count() == 1
+    _check(got, ref, "bf16")
+
+
 @pytest.mark.parametrize("idx", [0, 1, 3, 4], ids=[synth.CONFIGS[i].name for i in (0, 1, 3, 4)])
 def test_gradient_benchmark_config_full_size(oracle, idx):
     """Configurations at full size through the entry point the benchmark times; the oracle (which keeps every state of
