@@ -195,7 +195,12 @@ int vig_bigla_fwd_blend_bf16(const void* q, const void* k, const void* v,
  * How: dv is the forward pass itself on (k, q, d_out) with the gates moved by one token (the tensor-core kernels for
  * the bf16 head sizes they cover); dq, dk and the gate gradients come from two fp32 walks over the sequence per unit
  * on the CUDA cores (states in registers), with the gate gradients as running sums of q * dq - k * dk per direction.
- * Scratch (the moved gates, 8 L dk bytes per unit of partial results) comes from the library's pool, stream-ordered.
+ * Calls with few units and long sequences (fewer than two units per SM, 128 tokens or more) cut every sequence into
+ * segments that are walked in parallel: a first launch finds what each segment adds to the four states, a fold carries
+ * the states across segments, the walks start from them, and a last launch adds the later segments' sums to the gate
+ * gradients (vig_t-like 1024 x 1024 inputs, 32 units of 4096 tokens: 2.19 ms -> 0.55 ms).
+ * Scratch (the moved gates, 8 L dk bytes per unit of partial results, the segments' states) comes from the library's
+ * pool, stream-ordered.
  * Head sizes: dk <= 128, dv <= 128, and whatever the forward entry point of the same type takes.
  * Errors: NULL_POINTER, BAD_DIM, MISALIGNED, UNSUPPORTED, CUDA. */
 int vig_bigla_bwd_bf16(const void* q, const void* k, const void* v,

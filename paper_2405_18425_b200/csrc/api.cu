@@ -204,7 +204,9 @@ static int bwd_impl(const void* q, const void* k, const void* v, const void* la_
     const long long units = (long long)B * H;
     const size_t gate_bytes = ((size_t)units * L * dk * sizeof(T) + 255) / 256 * 256;
     char* scratch = nullptr;
-    if (pool_alloc((void**)&scratch, 2 * gate_bytes + bwd_scratch_bytes(units, L, dk), stream) != cudaSuccess) return VIG_ERR_CUDA;
+    const size_t walk_bytes = bwd_scratch_bytes(units, L, dk, dv);
+    if (walk_bytes == 0) return VIG_ERR_CUDA;
+    if (pool_alloc((void**)&scratch, 2 * gate_bytes + walk_bytes, stream) != cudaSuccess) return VIG_ERR_CUDA;
     T *sf = (T*)scratch, *sb = (T*)(scratch + gate_bytes);
     if (launch_shift_gates<T>((const T*)la_f, (const T*)la_b, sf, sb, units, L, dk, stream) != cudaSuccess) st = VIG_ERR_CUDA;
     if (st == VIG_OK) {

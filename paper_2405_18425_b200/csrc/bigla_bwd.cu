@@ -35,9 +35,14 @@ template <typename T>
 struct BwdArgs {
     const T *q, *k, *v, *la_f, *la_b, *g;
     T *dq, *dkey, *dla_f, *dla_b;
-    float* scratch;   // [units][L][dk][2] fp32: (dq>, dk<) between the two walks
+    float* scratch;   // [units][L][dk][2] fp32: (dq>, dk<) between the two walks (then the local gate sums of a segmented call)
+    // Segmented call (few units, long sequences): a block walks one segment of seg_len tokens.  states: [units][nseg][4]
+    // [dk][CG CN] fp32 - S>, Z<, S<, Z> of a segment run from zero, replaced by the states entering the segment; decay:
+    // [units][nseg][4][dk] - the products of the gates over the segment; totals: [units][nseg][2][dk] - the segment's sums of
+    // E> and E<.  All NULL / nseg = 1 for the call that walks whole units.
+    float *states, *decay, *totals;
     long long units;
-    int L, dk, dv;
+    int L, dk, dv, nseg, seg_len;
 };
 
 // Shared memory of a block.  rows: state rows it holds (threads / CG, >= dk; the padded rows and columns work on
@@ -83,7 +88,9 @@ constexpr int bwd_min_blocks(int rows, int cg) { return rows > 0 ? 768 / (rows *
 // CG: threads (adjacent lanes) per state row, 2 or 4.  CN: columns of the state per thread (a multiple of 4).  ROWS: state
 // rows of the block (threads / CG) when known at compile time - every shared-memory offset is then an immediate - or 0
 // for any block size.
-template <typename T, int CN, int ROWS, int CG>
+// SUMMARY: the first launch of a segmented call - the four states of every segment run from zero and the products of their
+// gates (state updates only, nothing else is read or written).
+template <typename T, int CN, int ROWS, int CG, bool SUMMARY>
 __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS, CG)) bigla_bwd_kernel(BwdArgs<T> a) {
     constexpr int kBwdCG = CG;
     static_assert(CN % 4 == 0, "columns per thread come in 16-byte pieces");
@@ -109,10 +116,13 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
     const bool ahead = (dk * sizeof(T)) % 16 == 0 && (dv * sizeof(T)) % 16 == 0;
     for (size_t x = tid; x < bwd_stage_floats(rows, CN, CG); x += nt) bw_smem[x] = 0.f;   // the padding stays zero
     __syncthreads();
-    const int nchunk = (L + kBwdTT - 1) / kBwdTT;
     const int st_r = tid % rows, st_t = tid / rows;   // staging: thread = one key dimension of every fourth token
+    const bool segmented = a.states != nullptr;
 
-    for (long long unit = blockIdx.x; unit < a.units; unit += gridDim.x) {
+    for (long long w = blockIdx.x; w < a.units * a.nseg; w += gridDim.x) {
+        const long long unit = w / a.nseg;
+        const int s0 = (int)(w % a.nseg) * a.seg_len, s1 = min(L, s0 + a.seg_len);   // this block's tokens [s0, s1)
+        const int nchunk = (s1 - s0 + kBwdTT - 1) / kBwdTT;
         const size_t ok = (size_t)unit * L * dk, ov = (size_t)unit * L * dv;
         float2* sc = reinterpret_cast<float2*>(a.scratch) + ok;   // [L][dk] pairs (dq>, dk<)
         for (int walk = 0; walk < 2; ++walk) {
@@ -123,10 +133,21 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
 #pragma unroll
             for (int c = 0; c < CN / 2; ++c) S[c] = Z[c] = 0ull;   // (+0, +0)
             float run_f = 0.f, run_b = 0.f;   // running sums of E> and E< (descending walk)
+            float prod_s = 1.f, prod_z = 1.f;   // SUMMARY: products of the gates of S and of Z over the segment
+            const size_t st_base = ((size_t)w * 4 + (walk == 0 ? 0 : 2)) * dk;   // kinds: S> 0, Z< 1, S< 2, Z> 3
+            if (!SUMMARY && segmented && i < dk) {   // the states that enter this segment
+                const float* ps = a.states + (st_base + i) * (CG * CN) + cg * CN;
+                const float* pz = ps + (size_t)dk * (CG * CN);
+#pragma unroll
+                for (int c = 0; c < CN / 2; ++c) {
+                    S[c] = pack2(ps[2 * c], ps[2 * c + 1]);
+                    Z[c] = pack2(pz[2 * c], pz[2 * c + 1]);
+                }
+            }
             // sixteen tokens of every input on their way into the landing zone (thread = 16-byte pieces)
             auto fetch = [&](int cc) {
-                const int t0 = (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
-                const int nv = min(kBwdTT, L - t0);
+                const int t0 = s0 + (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
+                const int nv = min(kBwdTT, s1 - t0);
                 const int pk = nv * dk * (int)sizeof(T) / 16, pv = nv * dv * (int)sizeof(T) / 16, row16 = dk * (int)sizeof(T) / 16;
                 const char* gk = reinterpret_cast<const char*>(a.k + ok + (size_t)t0 * dk);
                 const char* gq = reinterpret_cast<const char*>(a.q + ok + (size_t)t0 * dk);
@@ -145,7 +166,7 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                     cp_async16(reinterpret_cast<char*>(raw_v) + 16 * x, gv + 16 * x);
                     cp_async16(reinterpret_cast<char*>(raw_g) + 16 * x, gg + 16 * x);
                 }
-                if (walk == 1) {
+                if (walk == 1 && !SUMMARY) {
                     const char* gx = reinterpret_cast<const char*>(sc + (size_t)t0 * dk);
                     for (int x = tid; x < nv * dk / 2; x += nt) cp_async16(reinterpret_cast<char*>(raw_x) + 16 * x, gx + 16 * x);
                 }
@@ -163,7 +184,7 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         r4.z = expf(rec_to_float(s_[e]));
                         r4.w = (tp >= 0 && tp < L) ? expf(rec_to_float(z_[e])) : 0.f;
                         rowd[tt * rows + st_r] = r4;
-                        if (walk == 1) xd[tt * rows + st_r] = x_[e];
+                        if (walk == 1 && !SUMMARY) xd[tt * rows + st_r] = x_[e];
                     }
                 }
                 int tt = 0, j = tid;
@@ -189,7 +210,7 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                     const bool zin = tp >= 0 && tp < L;
 #pragma unroll
                     for (int u = 0; u < 4; ++u) rowd[tt * rows + r0 + u] = make_float4(kf[u], qf[u], expf(sf[u]), zin ? expf(zf[u]) : 0.f);
-                    if (walk == 1) {
+                    if (walk == 1 && !SUMMARY) {
                         const float4 xa = *reinterpret_cast<const float4*>(raw_x + e), xb = *reinterpret_cast<const float4*>(raw_x + e + 2);
                         float4* xo = reinterpret_cast<float4*>(xd + tt * rows + r0);
                         xo[0] = xa;
@@ -208,8 +229,8 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
             };
             if (ahead) fetch(0);
             for (int cc = 0; cc < nchunk; ++cc) {
-                const int t0 = (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
-                const int nv = min(kBwdTT, L - t0);
+                const int t0 = s0 + (walk == 0 ? cc : nchunk - 1 - cc) * kBwdTT;
+                const int nv = min(kBwdTT, s1 - t0);
                 if (ahead) {
                     asm volatile("cp.async.wait_group 0;" ::: "memory");
                     __syncthreads();   // everybody's pieces have landed (and the results of the chunk before are stored)
@@ -238,6 +259,21 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         const ulonglong2* vr = reinterpret_cast<const ulonglong2*>(vp);   // two pairs each
                         const ulonglong2* gr = reinterpret_cast<const ulonglong2*>(gp);
                         const f32x2 ds2 = pack2(r4.z, r4.z), dz2 = pack2(r4.w, r4.w), kq2 = pack2(r4.x, r4.x), hq2 = pack2(hq, hq);
+                        if constexpr (SUMMARY) {
+#pragma unroll
+                            for (int c4 = 0; c4 < CN / 4; ++c4) {
+                                const ulonglong2 v4 = vr[c4], g4 = gr[c4];
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const int c = 2 * c4 + h;
+                                    S[c] = ffma2(ds2, S[c], fmul2(kq2, h == 0 ? v4.x : v4.y));
+                                    Z[c] = ffma2(dz2, Z[c], fmul2(hq2, h == 0 ? g4.x : g4.y));
+                                }
+                            }
+                            prod_s *= r4.z;
+                            prod_z *= r4.w;
+                            continue;
+                        }
                         f32x2 aq[2] = {0ull, 0ull}, ak[2] = {0ull, 0ull};
 #pragma unroll
                         for (int c4 = 0; c4 < CN / 4; ++c4) {
@@ -265,12 +301,13 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         } else {
                             const float2 x2 = *xp;   // dq>_t, dk<_t;  accq = dq<_t, acck = dk>_t
                             run_f += r4.y * x2.x - r4.x * acck;
-                            // dq, dk, the sum over m >= t of E>_m, minus the sum over m > t of E<_m
+                            // dq, dk, the sum over m >= t of E>_m, minus the sum over m > t of E<_m (within the block's tokens)
                             if (cg == 0) sts128_untracked(op, x2.x + accq, acck + x2.y, run_f, -run_b);
                             run_b += r4.y * accq - r4.x * x2.y;
                         }
                     }
                 }
+                if constexpr (SUMMARY) continue;   // nothing to store per token (the barrier at the top of the loop orders the staging)
                 __syncthreads();
                 if (ahead) {   // four key dimensions of a token per thread: 8- or 16-byte stores
                     const int qk = dk / 4;
@@ -290,8 +327,14 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         } else {
                             store4(a.dq + ok + gi, o[0]);
                             store4(a.dkey + ok + gi, o[1]);
-                            store4(a.dla_f + ok + gi, o[2]);
-                            store4(a.dla_b + ok + gi, o[3]);
+                            if (segmented) {   // the gate sums of this segment alone, in fp32 over the consumed pairs
+                                float4* so = reinterpret_cast<float4*>(sc + gi);
+                                so[0] = make_float4(o[2][0], o[3][0], o[2][1], o[3][1]);
+                                so[1] = make_float4(o[2][2], o[3][2], o[2][3], o[3][3]);
+                            } else {
+                                store4(a.dla_f + ok + gi, o[2]);
+                                store4(a.dla_b + ok + gi, o[3]);
+                            }
                         }
                     }
                 } else if (st_r < dk) {
@@ -303,14 +346,85 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         } else {
                             rec_store(a.dq + ok + gi, o4.x);
                             rec_store(a.dkey + ok + gi, o4.y);
-                            rec_store(a.dla_f + ok + gi, o4.z);
-                            rec_store(a.dla_b + ok + gi, o4.w);
+                            if (segmented) {
+                                sc[gi] = make_float2(o4.z, o4.w);
+                            } else {
+                                rec_store(a.dla_f + ok + gi, o4.z);
+                                rec_store(a.dla_b + ok + gi, o4.w);
+                            }
                         }
                     }
                 }
             }
+            if (SUMMARY && i < dk) {   // what the segment adds to each state, and by how much it shrinks what enters it
+                float* ps = a.states + (st_base + i) * (CG * CN) + cg * CN;
+                float* pz = ps + (size_t)dk * (CG * CN);
+#pragma unroll
+                for (int c = 0; c < CN / 2; ++c) {
+                    unpack2(S[c], ps[2 * c], ps[2 * c + 1]);
+                    unpack2(Z[c], pz[2 * c], pz[2 * c + 1]);
+                }
+                if (cg == 0) {
+                    a.decay[st_base + i] = prod_s;
+                    a.decay[st_base + dk + i] = prod_z;
+                }
+            }
+            if (!SUMMARY && segmented && walk == 1 && cg == 0 && i < dk) {
+                a.totals[((size_t)w * 2) * dk + i] = run_f;
+                a.totals[((size_t)w * 2 + 1) * dk + i] = run_b;
+            }
             __syncthreads();   // the scratch of the ascending walk is read back by other threads
         }
+    }
+}
+
+// Second launch of a segmented call: the states that enter each segment, X_in(s + 1) = D(s) X_in(s) + X(s) walking up for
+// S> and Z<, X_in(s - 1) = D(s) X_in(s) + X(s) walking down for S< and Z>, written over the segments' own states.
+// Thread = four columns of one state row of one unit.
+__global__ void __launch_bounds__(256) bwd_fold_kernel(float* states, const float* decay, long long units, int nseg, int dk, int cols) {
+    const int c4 = cols / 4;
+    const long long n = units * dk * c4;
+    for (long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x; x < n; x += (long long)gridDim.x * blockDim.x) {
+        const int col = (int)(x % c4) * 4, i = (int)((x / c4) % dk);
+        const long long unit = x / ((long long)c4 * dk);
+#pragma unroll
+        for (int kind = 0; kind < 4; ++kind) {
+            float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int n2 = 0; n2 < nseg; ++n2) {
+                const int sg = kind < 2 ? n2 : nseg - 1 - n2;
+                const size_t row = (((size_t)unit * nseg + sg) * 4 + kind) * dk + i;
+                float4* p = reinterpret_cast<float4*>(states + row * cols + col);
+                const float4 own = *p;
+                const float d = decay[row];
+                *p = carry;
+                carry = make_float4(fmaf(d, carry.x, own.x), fmaf(d, carry.y, own.y), fmaf(d, carry.z, own.z), fmaf(d, carry.w, own.w));
+            }
+        }
+    }
+}
+
+// Last launch of a segmented call: the gate gradients of a token are its segment's local sums plus what the segments
+// walked before it (the later ones) add: dlog alpha>_t = local + sum_{s' > s} total>(s'), dlog alpha<_t = local - sum_{s' > s}
+// total<(s').  Block = one segment of one unit.
+template <typename T>
+__global__ void __launch_bounds__(256) bwd_finish_kernel(const float2* local, const float* totals, T* dla_f, T* dla_b, int L, int dk, int nseg,
+                                                         int seg_len) {
+    extern __shared__ float off[];   // [2][dk]
+    const long long w = blockIdx.x, unit = w / nseg;
+    const int sg = (int)(w % nseg), s0 = sg * seg_len, s1 = min(L, s0 + seg_len);
+    for (int x = threadIdx.x; x < 2 * dk; x += blockDim.x) {
+        const int which = x / dk, i = x - which * dk;
+        float acc = 0.f;
+        for (int s2 = nseg - 1; s2 > sg; --s2) acc += totals[(((size_t)unit * nseg + s2) * 2 + which) * dk + i];   // in walking order
+        off[x] = which == 0 ? acc : -acc;
+    }
+    __syncthreads();
+    const size_t base = ((size_t)unit * L + s0) * dk;
+    for (int x = threadIdx.x; x < (s1 - s0) * dk; x += blockDim.x) {
+        const float2 l = local[base + x];
+        const int i = x % dk;
+        rec_store(dla_f + base + x, l.x + off[i]);
+        rec_store(dla_b + base + x, l.y + off[dk + i]);
     }
 }
 
@@ -331,8 +445,8 @@ __global__ void __launch_bounds__(256) shift_gates_kernel(const V* __restrict__ 
     }
 }
 
-template <typename T, int CN, int ROWS, int CG>
-cudaError_t launch_bwd_t(const BwdArgs<T>& a, int threads, int sms, cudaStream_t stream) {
+template <typename T, int CN, int ROWS, int CG, bool SUMMARY>
+cudaError_t launch_bwd_kernel(const BwdArgs<T>& a, int threads, int sms, cudaStream_t stream) {
     const size_t smem = bwd_smem_bytes(threads / CG, CN, CG, a.dk, a.dv, sizeof(T));
     static std::atomic<bool> configured[64];
     int dev = 0;
@@ -340,12 +454,35 @@ cudaError_t launch_bwd_t(const BwdArgs<T>& a, int threads, int sms, cudaStream_t
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!configured[dev].load(std::memory_order_acquire)) {
-        if ((e = cudaFuncSetAttribute(bigla_bwd_kernel<T, CN, ROWS, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess)
+        if ((e = cudaFuncSetAttribute(bigla_bwd_kernel<T, CN, ROWS, CG, SUMMARY>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) !=
+            cudaSuccess)
             return e;
         configured[dev].store(true, std::memory_order_release);
     }
-    long long grid = a.units < 32LL * sms ? a.units : 32LL * sms;
-    bigla_bwd_kernel<T, CN, ROWS, CG><<<(unsigned)grid, threads, smem, stream>>>(a);
+    const long long work = a.units * a.nseg;
+    long long grid = work < 32LL * sms ? work : 32LL * sms;
+    bigla_bwd_kernel<T, CN, ROWS, CG, SUMMARY><<<(unsigned)grid, threads, smem, stream>>>(a);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// The walks of a call: one launch over whole units, or - segmented - the segments' own states, the fold that turns them
+// into the states entering each segment, the walks proper from those states, and the gate gradients put together.
+template <typename T, int CN, int ROWS, int CG>
+cudaError_t launch_bwd_t(const BwdArgs<T>& a, int threads, int sms, cudaStream_t stream) {
+    if (a.nseg == 1) return launch_bwd_kernel<T, CN, ROWS, CG, false>(a, threads, sms, stream);
+    cudaError_t e = launch_bwd_kernel<T, CN, ROWS, CG, true>(a, threads, sms, stream);
+    if (e != cudaSuccess) return e;
+    const int cols = CG * CN;
+    const long long n = a.units * a.dk * (cols / 4);
+    long long blocks = (n + 255) / 256;
+    if (blocks > 8LL * sms) blocks = 8LL * sms;
+    bwd_fold_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a.states, a.decay, a.units, a.nseg, a.dk, cols);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_bwd_kernel<T, CN, ROWS, CG, false>(a, threads, sms, stream)) != cudaSuccess) return e;
+    bwd_finish_kernel<T><<<(unsigned)(a.units * a.nseg), 256, 2 * a.dk * sizeof(float), stream>>>(
+        reinterpret_cast<const float2*>(a.scratch), a.totals, a.dla_f, a.dla_b, a.L, a.dk, a.nseg, a.seg_len);
     count_launch();
     return cudaGetLastError();
 }
@@ -361,6 +498,27 @@ int bwd_cn(int dv, int cg) {   // columns per thread: the instantiated size that
     return cn <= 8 ? 8 : (cn <= 12 ? 12 : (cn <= 16 ? 16 : (cn <= 24 ? 24 : 32)));
 }
 
+// Few units and long sequences: the sequence is cut into segments so that about five blocks per SM walk at once (a lone
+// block per SM needs about 550 cycles per token).  Segments are multiples of the staging group and at least 64 tokens.
+void bwd_plan(long long units, int L, int sms, int* nseg, int* seg_len) {
+    *nseg = 1;
+    *seg_len = L > 0 ? L : 1;
+    if (units >= 2LL * sms || L < 128) return;
+    long long want = (5LL * sms + units - 1) / units;
+    if (want > L / 64) want = L / 64;
+    if (want < 2) return;
+    const int len = (int)(((L + want - 1) / want + kBwdTT - 1) / kBwdTT * kBwdTT);
+    *seg_len = len;
+    *nseg = (L + len - 1) / len;
+}
+
+cudaError_t sm_count_of_device(int* sms) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    return cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev);
+}
+
 }  // namespace
 
 bool bwd_supported(int dk, int dv) {
@@ -369,7 +527,23 @@ bool bwd_supported(int dk, int dv) {
     return bwd_smem_bytes(threads / cg, bwd_cn(dv, cg), cg, dk, dv, 4) <= 200 * 1024;
 }
 
-size_t bwd_scratch_bytes(long long units, int L, int dk) { return (size_t)units * 2 * L * dk * sizeof(float); }
+// Scratch of the walks, in floats: the per-token pairs, then (segmented calls) the segment states, gate products and sums.
+static void bwd_scratch_layout(long long units, int L, int dk, int dv, int nseg, size_t* pairs, size_t* states, size_t* decay, size_t* totals) {
+    const int cg = bwd_cg(dv), cols = cg * bwd_cn(dv, cg);
+    *pairs = ((size_t)units * 2 * L * dk + 63) / 64 * 64;
+    *states = nseg > 1 ? (size_t)units * nseg * 4 * dk * cols : 0;
+    *decay = nseg > 1 ? ((size_t)units * nseg * 4 * dk + 63) / 64 * 64 : 0;
+    *totals = nseg > 1 ? (size_t)units * nseg * 2 * dk : 0;
+}
+
+size_t bwd_scratch_bytes(long long units, int L, int dk, int dv) {
+    int sms = 0, nseg, seg_len;
+    if (sm_count_of_device(&sms) != cudaSuccess) return 0;
+    bwd_plan(units, L, sms, &nseg, &seg_len);
+    size_t p, st, de, to;
+    bwd_scratch_layout(units, L, dk, dv, nseg, &p, &st, &de, &to);
+    return (p + st + de + to) * sizeof(float);
+}
 
 template <typename T>
 cudaError_t launch_shift_gates(const T* la_f, const T* la_b, T* out_f, T* out_b, long long units, int L, int dk, cudaStream_t stream) {
@@ -389,11 +563,15 @@ cudaError_t launch_shift_gates(const T* la_f, const T* la_b, T* out_f, T* out_b,
 template <typename T>
 cudaError_t launch_bigla_bwd(const T* q, const T* k, const T* v, const T* la_f, const T* la_b, const T* d_out, T* dq, T* dk_out, T* dla_f,
                              T* dla_b, float* scratch, long long units, int L, int dk, int dv, cudaStream_t stream) {
-    int dev = 0, sms = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    int sms = 0, nseg, seg_len;
+    cudaError_t e = sm_count_of_device(&sms);
     if (e != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    BwdArgs<T> a{q, k, v, la_f, la_b, d_out, dq, dk_out, dla_f, dla_b, scratch, units, L, dk, dv};
+    bwd_plan(units, L, sms, &nseg, &seg_len);
+    size_t p, st, de, to;
+    bwd_scratch_layout(units, L, dk, dv, nseg, &p, &st, &de, &to);
+    BwdArgs<T> a{q, k, v, la_f, la_b, d_out, dq, dk_out, dla_f, dla_b, scratch,
+                 nseg > 1 ? scratch + p : nullptr, nseg > 1 ? scratch + p + st : nullptr, nseg > 1 ? scratch + p + st + de : nullptr,
+                 units, L, dk, dv, nseg, seg_len};
     const int cg = bwd_cg(dv), threads = bwd_threads(dk, cg), cn = bwd_cn(dv, cg), rows = threads / cg;
 #define VIG_BWD_CASE(CN_, ROWS_, CG_) \
     if (cn == CN_ && cg == CG_ && (ROWS_ == 0 || rows == ROWS_)) return launch_bwd_t<T, CN_, ROWS_, CG_>(a, threads, sms, stream);

@@ -68,7 +68,7 @@ cudaError_t launch_bigla_umma_long(const __nv_bfloat16* q, const __nv_bfloat16* 
 // ---- gradient of the forward pass with respect to q, k and the log gates (fp32 recurrences on the CUDA cores); the
 // gradient with respect to v is the forward pass on (k, q, d_out) with the gates from launch_shift_gates ----
 bool bwd_supported(int dk, int dv);
-size_t bwd_scratch_bytes(long long units, int L, int dk);
+size_t bwd_scratch_bytes(long long units, int L, int dk, int dv);   // 0: the device could not be queried
 template <typename T>
 cudaError_t launch_shift_gates(const T* la_f, const T* la_b, T* out_f, T* out_b, long long units, int L, int dk, cudaStream_t stream);
 template <typename T>
