@@ -470,7 +470,8 @@ def run_gpu(args, cfg):
 
     # ---- every bf16 workload, so that one record carries all shapes (shorter regions for the others) ----
     per = {cfg.name: {"us_per_call": ms_per_step * 1e3, "unfused_us_per_call": float(np.median(unfused_ms)) * 1e3,
-                      "scan_only_us": scan_us, "roofline": {"frac": line["roofline"]["frac"], "traffic": line["roofline"]["traffic"]},
+                      "scan_only_us": scan_us, "bwd_us_per_call": bwd_us,
+                      "roofline": {"frac": line["roofline"]["frac"], "traffic": line["roofline"]["traffic"]},
                       "B": cfg.B, "H": cfg.H, "L": cfg.L, "dk": cfg.dk, "dv": cfg.dv}}
     del w
     torch.cuda.empty_cache()
@@ -483,9 +484,10 @@ def run_gpu(args, cfg):
             u_ms, _, _ = wo.time(wo.unfused, k_small, args.warmup, 10.0)
             s_ms, _, _ = wo.time(wo.scan, k_small, args.warmup, 10.0)
             s_us = float(np.median(s_ms)) * 1e3
+            b_ms, _, _ = wo.time(wo.bwd, min(k_small, 20), args.warmup, 5.0)   # the gradient call (log alpha is in place)
             r = roofline_of(other, s_us, "vig_bigla_fwd_bf16")
             per[other.name] = {"us_per_call": float(np.median(f_ms)) * 1e3, "unfused_us_per_call": float(np.median(u_ms)) * 1e3,
-                               "scan_only_us": s_us, "roofline": {"frac": r["frac"], "traffic": r["traffic"]},
+                               "scan_only_us": s_us, "bwd_us_per_call": float(np.median(b_ms)) * 1e3, "roofline": {"frac": r["frac"], "traffic": r["traffic"]},
                                "B": other.B, "H": other.H, "L": other.L, "dk": other.dk, "dv": other.dv}
             del wo
             torch.cuda.empty_cache()
