@@ -112,6 +112,12 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
     T* raw_v = raw_z + kBwdTT * dk;
     T* raw_g = raw_v + kBwdTT * dv;
     float2* raw_x = reinterpret_cast<float2*>(raw_g + kBwdTT * dv);
+    // The instances for the paper's head sizes (bf16, dv = CG CN exactly, whole 16-byte rows) read v and d_out in the walk
+    // straight from the landing zone, as bf16: half the shared-memory traffic of the walk, which is what bounds it.  The
+    // landing zone of v and d_out then has a second buffer (in place of the fp32 staging of the two).
+    constexpr bool kVG16 = ROWS != 0 && sizeof(T) == 2;
+    T* raw_v1 = reinterpret_cast<T*>(vs);
+    T* raw_g1 = raw_v1 + kBwdTT * dv;
     // Rows of whole 16-byte pieces: the next sixteen tokens are copied asynchronously while these are worked on.
     const bool ahead = (dk * sizeof(T)) % 16 == 0 && (dv * sizeof(T)) % 16 == 0;
     for (size_t x = tid; x < bwd_stage_floats(rows, CN, CG); x += nt) bw_smem[x] = 0.f;   // the padding stays zero
@@ -162,9 +168,11 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                 }
                 const char* gv = reinterpret_cast<const char*>(a.v + ov + (size_t)t0 * dv);
                 const char* gg = reinterpret_cast<const char*>(a.g + ov + (size_t)t0 * dv);
+                char* dv_ = reinterpret_cast<char*>(kVG16 && (cc & 1) ? raw_v1 : raw_v);
+                char* dg_ = reinterpret_cast<char*>(kVG16 && (cc & 1) ? raw_g1 : raw_g);
                 for (int x = tid; x < pv; x += nt) {
-                    cp_async16(reinterpret_cast<char*>(raw_v) + 16 * x, gv + 16 * x);
-                    cp_async16(reinterpret_cast<char*>(raw_g) + 16 * x, gg + 16 * x);
+                    cp_async16(dv_ + 16 * x, gv + 16 * x);
+                    cp_async16(dg_ + 16 * x, gg + 16 * x);
                 }
                 if (walk == 1 && !SUMMARY) {
                     const char* gx = reinterpret_cast<const char*>(sc + (size_t)t0 * dk);
@@ -217,7 +225,7 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         xo[1] = xb;
                     }
                 }
-                for (int x = tid; x < nv * qv; x += nt) {
+                for (int x = tid; x < (kVG16 ? 0 : nv * qv); x += nt) {   // (kVG16: v and d_out stay where they landed)
                     const int tt = x / qv, j0 = (x - tt * qv) * 4;
                     const int at = tt * cols + (j0 / CN) * (CN + 4) + j0 % CN;
                     float f[4];
@@ -249,25 +257,41 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                     const float2* xp = xd + (walk == 0 ? 0 : nv - 1) * rows + i;
                     float4* op = rowd + (walk == 0 ? 0 : nv - 1) * rows + i;   // the record is replaced by the results (the lanes of a
                                                                                 // row read it in the same instruction, before this lane writes)
-                    const float* vp = vs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
-                    const float* gp = gs + (walk == 0 ? 0 : nv - 1) * cols + cg * (CN + 4);
-                    const int srow = step * rows, scol = step * cols;
+                    const int first = walk == 0 ? 0 : nv - 1;
+                    // this thread's columns of v and d_out, token by token: fp32 staging, or (kVG16) the bf16 rows as they landed
+                    const char* vp = kVG16 ? reinterpret_cast<const char*>(((cc & 1) ? raw_v1 : raw_v) + first * dv + cg * CN)
+                                           : reinterpret_cast<const char*>(vs + first * cols + cg * (CN + 4));
+                    const char* gp = kVG16 ? reinterpret_cast<const char*>(((cc & 1) ? raw_g1 : raw_g) + first * dv + cg * CN)
+                                           : reinterpret_cast<const char*>(gs + first * cols + cg * (CN + 4));
+                    const int srow = step * rows, scol = step * (kVG16 ? dv * 2 : cols * 4);   // bytes per token
+                    // four columns (two fp32 pairs) number c4 of the row at p
+                    auto quad = [&](const char* p, int c4, f32x2& lo, f32x2& hi) {
+                        if constexpr (kVG16) {
+                            const uint2 wv = reinterpret_cast<const uint2*>(p)[c4];   // a bf16 is the upper half of its fp32
+                            lo = pack2(__uint_as_float(wv.x << 16), __uint_as_float(wv.x & 0xffff0000u));
+                            hi = pack2(__uint_as_float(wv.y << 16), __uint_as_float(wv.y & 0xffff0000u));
+                        } else {
+                            const ulonglong2 q2 = reinterpret_cast<const ulonglong2*>(p)[c4];
+                            lo = q2.x;
+                            hi = q2.y;
+                        }
+                    };
 #pragma unroll 4
                     for (int n = 0; n < nv; ++n, rp += srow, xp += srow, op += srow, vp += scol, gp += scol) {
                         const float4 r4 = *rp;   // k, q, decay of S, decay of Z
                         const float hq = 0.5f * r4.y;
-                        const ulonglong2* vr = reinterpret_cast<const ulonglong2*>(vp);   // two pairs each
-                        const ulonglong2* gr = reinterpret_cast<const ulonglong2*>(gp);
                         const f32x2 ds2 = pack2(r4.z, r4.z), dz2 = pack2(r4.w, r4.w), kq2 = pack2(r4.x, r4.x), hq2 = pack2(hq, hq);
                         if constexpr (SUMMARY) {
 #pragma unroll
                             for (int c4 = 0; c4 < CN / 4; ++c4) {
-                                const ulonglong2 v4 = vr[c4], g4 = gr[c4];
+                                f32x2 vq[2], gq[2];
+                                quad(vp, c4, vq[0], vq[1]);
+                                quad(gp, c4, gq[0], gq[1]);
 #pragma unroll
                                 for (int h = 0; h < 2; ++h) {
                                     const int c = 2 * c4 + h;
-                                    S[c] = ffma2(ds2, S[c], fmul2(kq2, h == 0 ? v4.x : v4.y));
-                                    Z[c] = ffma2(dz2, Z[c], fmul2(hq2, h == 0 ? g4.x : g4.y));
+                                    S[c] = ffma2(ds2, S[c], fmul2(kq2, vq[h]));
+                                    Z[c] = ffma2(dz2, Z[c], fmul2(hq2, gq[h]));
                                 }
                             }
                             prod_s *= r4.z;
@@ -277,10 +301,12 @@ __global__ void __launch_bounds__(bwd_max_threads(ROWS, CG), bwd_min_blocks(ROWS
                         f32x2 aq[2] = {0ull, 0ull}, ak[2] = {0ull, 0ull};
 #pragma unroll
                         for (int c4 = 0; c4 < CN / 4; ++c4) {
-                            const ulonglong2 v4 = vr[c4], g4 = gr[c4];
+                            f32x2 vq[2], gq[2];
+                            quad(vp, c4, vq[0], vq[1]);
+                            quad(gp, c4, gq[0], gq[1]);
 #pragma unroll
                             for (int h = 0; h < 2; ++h) {
-                                const f32x2 vj = h == 0 ? v4.x : v4.y, gj = h == 0 ? g4.x : g4.y;
+                                const f32x2 vj = vq[h], gj = gq[h];
                                 const int c = 2 * c4 + h;
                                 S[c] = ffma2(ds2, S[c], fmul2(kq2, vj));   // S_t = a S + k^T v
                                 aq[h] = ffma2(S[c], gj, aq[h]);            // S_t g^T
@@ -574,7 +600,7 @@ cudaError_t launch_bigla_bwd(const T* q, const T* k, const T* v, const T* la_f, 
                  units, L, dk, dv, nseg, seg_len};
     const int cg = bwd_cg(dv), threads = bwd_threads(dk, cg), cn = bwd_cn(dv, cg), rows = threads / cg;
 #define VIG_BWD_CASE(CN_, ROWS_, CG_) \
-    if (cn == CN_ && cg == CG_ && (ROWS_ == 0 || rows == ROWS_)) return launch_bwd_t<T, CN_, ROWS_, CG_>(a, threads, sms, stream);
+    if (cn == CN_ && cg == CG_ && (ROWS_ == 0 || (dk == ROWS_ && dv == CG_ * CN_))) return launch_bwd_t<T, CN_, ROWS_, CG_>(a, threads, sms, stream);
     if constexpr (sizeof(T) == 2) {   // the head sizes of the paper's models: block shape known at compile time
         VIG_BWD_CASE(8, 16, 4) VIG_BWD_CASE(8, 24, 4) VIG_BWD_CASE(8, 32, 4)        // dv = 32; dk = 16, 24, 32
         VIG_BWD_CASE(12, 16, 4) VIG_BWD_CASE(12, 24, 4) VIG_BWD_CASE(12, 32, 4)     // dv = 48
