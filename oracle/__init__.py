@@ -9,6 +9,6 @@ from .oracle import (  # noqa: F401
     build_oracle,
     gate_prep,
 )
-from .backward import bigla_bwd  # noqa: F401
+from .backward import bigla_bwd, gate_prep_bwd  # noqa: F401
 from .locality import dwconv3x3, gate_blend  # noqa: F401
 from .quadratic import bigla_quadratic  # noqa: F401

@@ -61,3 +61,14 @@ def bigla_bwd(q, k, v, log_alpha_fwd, log_alpha_bwd, d_out):
     out = (fq + unflip(bq), fk + unflip(bk), fv + unflip(bv), fl, unflip(bl))
     shapes = (q.shape, k.shape, v.shape, laf.shape, lab.shape)
     return tuple(np.ascontiguousarray(x).reshape(s) for x, s in zip(out, shapes))
+
+
+def gate_prep_bwd(g, dlog_alpha, tau: float = 16.0):
+    """Gradient through the gate preparation log alpha = logsigmoid(g) / tau (Eq. 5 line 1):
+    dg = dlog_alpha * sigmoid(-g) / tau, since d/dg log(sigmoid(g)) = 1 - sigmoid(g).  fp64, shaped like g.
+    (exp is only taken of non-positive numbers.)"""
+    g = np.asarray(g, dtype=np.float64)
+    d = np.asarray(dlog_alpha, dtype=np.float64)
+    e = np.exp(-np.abs(g))
+    sig_neg = np.where(g >= 0, e / (1.0 + e), 1.0 / (1.0 + e))   # sigmoid(-g)
+    return d * sig_neg / float(tau)

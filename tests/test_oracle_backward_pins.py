@@ -10,7 +10,9 @@ import numpy as np
 import pytest
 import torch
 
-from oracle.backward import bigla_bwd
+import mpmath
+
+from oracle.backward import bigla_bwd, gate_prep_bwd
 
 
 def _rand(seed, B=1, H=2, L=6, dk=3, dv=2, gate_scale=1.0):
@@ -155,3 +157,39 @@ def test_planted_mistake_in_gradient_is_caught(fwd, mistake):
         except AssertionError:
             failed.append(pin.__name__)
     assert failed, f"no pin catches {mistake}"
+
+
+# ----------------------------------------------------------------------------------------------
+# Gradient through the gate preparation (Eq. 5 line 1)
+# ----------------------------------------------------------------------------------------------
+
+def _pins_gate_prep_bwd(fn, oracle):
+    r = np.random.default_rng(31)
+    g = np.concatenate([r.standard_normal(40) * 3, [-30.0, -1.0, 0.0, 1.0, 30.0]])
+    d = r.standard_normal(g.size)
+    for tau in (16.0, 3.0):
+        got = fn(g, d, tau)
+        h = 1e-6
+        num = (oracle.gate_prep(g + h, tau) - oracle.gate_prep(g - h, tau)) / (2 * h)   # the pinned forward oracle
+        np.testing.assert_allclose(got, d * num, rtol=1e-8, atol=1e-10)
+        np.testing.assert_allclose(fn(np.zeros(3), np.ones(3), tau), 0.5 / tau, rtol=1e-15)         # sigmoid(0) = 1/2
+        np.testing.assert_allclose(fn(g, np.ones_like(g), tau) + fn(-g, np.ones_like(g), tau), 1.0 / tau, rtol=1e-14)   # sigmoid(g) + sigmoid(-g) = 1
+    assert fn(np.array([800.0]), np.array([1.0]), 1.0)[0] == 0.0 and fn(np.array([-800.0]), np.array([1.0]), 1.0)[0] == 1.0
+    mpmath.mp.dps = 50
+    for gg in (-7.5, -0.3, 2.25, 11.0):
+        ref = mpmath.mpf(3) / (1 + mpmath.e ** mpmath.mpf(gg)) / 16
+        assert abs(fn(np.array([gg]), np.array([3.0]), 16.0)[0] - float(ref)) < 1e-16
+
+
+def test_gate_prep_gradient_oracle_pins(oracle):
+    _pins_gate_prep_bwd(gate_prep_bwd, oracle)
+
+
+@pytest.mark.parametrize("wrong", [
+    lambda g, d, tau: gate_prep_bwd(g, d, tau) * tau,                 # the temperature forgotten
+    lambda g, d, tau: gate_prep_bwd(-g, d, tau),                      # sigmoid(g) instead of 1 - sigmoid(g)
+    lambda g, d, tau: gate_prep_bwd(g, d, tau) * (1 - gate_prep_bwd(g, np.ones_like(g), 1.0)),   # the derivative of sigmoid, not of its logarithm
+], ids=["no_tau", "wrong_sign", "sigmoid_derivative"])
+def test_planted_mistake_in_gate_prep_gradient_is_caught(oracle, wrong):
+    with pytest.raises(AssertionError):
+        _pins_gate_prep_bwd(wrong, oracle)
