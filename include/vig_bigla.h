@@ -190,7 +190,7 @@ int vig_bigla_fwd_blend_bf16(const void* q, const void* k, const void* v,
  * the reverse-mode adjoint of Eq. 6 as it stands.  For d_out = dLoss/d_out [B,H,L,dv] the call writes
  *   dq, dk_out [B,H,L,dk], dv_out [B,H,L,dv], dlog_alpha_fwd, dlog_alpha_bwd [B,H,L,dk]
  * (gradients with respect to the LOG gates as passed to the forward call; a caller that feeds gate logits g chains
- * dg = dlog_alpha * (1 - sigmoid(g)) / tau, Eq. 5 line 1).  All device pointers of the call's element type, contiguous,
+ * them through vig_gate_prep_bwd_* below).  All device pointers of the call's element type, contiguous,
  * 16-byte aligned; inputs are not written; outputs must not overlap inputs or one another.
  * How: dv is the forward pass itself on (k, q, d_out) with the gates moved by one token (the tensor-core kernels for
  * the bf16 head sizes they cover); dq, dk and the gate gradients come from two fp32 walks over the sequence per unit
@@ -211,6 +211,15 @@ int vig_bigla_bwd_f32(const void* q, const void* k, const void* v,
                       const void* log_alpha_fwd, const void* log_alpha_bwd, const void* d_out,
                       void* dq, void* dk_out, void* dv_out, void* dlog_alpha_fwd, void* dlog_alpha_bwd,
                       int B, int H, int L, int dk, int dv, void* stream);
+
+/* vig_gate_prep_bwd_*: the gradient through the gate preparation (Eq. 5 line 1), for callers whose parameters sit
+ * behind the gate logits: dg = dlog_alpha * sigmoid(-g) / tau (d/dg log sigmoid(g) = 1 - sigmoid(g)), both directions
+ * in one launch, fp32 arithmetic.  g_*, dlog_alpha_*, dg_*: [B,H,L,dk] of the call's element type, 16-byte aligned;
+ * dg_* may be the dlog_alpha_* buffers (in place).  Errors: NULL_POINTER, BAD_DIM, MISALIGNED, CUDA. */
+int vig_gate_prep_bwd_bf16(const void* g_fwd, const void* g_bwd, const void* dlog_alpha_fwd, const void* dlog_alpha_bwd,
+                           void* dg_fwd, void* dg_bwd, int B, int H, int L, int dk, float tau, void* stream);
+int vig_gate_prep_bwd_f32(const void* g_fwd, const void* g_bwd, const void* dlog_alpha_fwd, const void* dlog_alpha_bwd,
+                          void* dg_fwd, void* dg_bwd, int B, int H, int L, int dk, float tau, void* stream);
 
 /* ---- Whole path on HOST buffers -------------------------------------------------------------------
  * Gate preparation followed by the BiGLA forward (Eq. 5 line 1 + Eq. 6) for callers whose data

@@ -18,6 +18,7 @@ from .binding import (  # noqa: F401
     vig_bigla_fwd_gates_bf16,
     vig_bigla_fwd_blend_bf16,
     vig_bigla_bwd,
+    vig_gate_prep_bwd,
     vig_dwconv3x3,
     vig_gate_blend,
     vig_bigla_fwd_host,

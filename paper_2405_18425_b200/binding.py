@@ -62,6 +62,9 @@ def load() -> ctypes.CDLL:
         for name in ("vig_bigla_bwd_bf16", "vig_bigla_bwd_f32"):
             getattr(lib, name).argtypes = [vp] * 11 + [ci] * 5 + [vp]
             getattr(lib, name).restype = ci
+        for name in ("vig_gate_prep_bwd_bf16", "vig_gate_prep_bwd_f32"):
+            getattr(lib, name).argtypes = [vp] * 6 + [ci] * 4 + [cf, vp]
+            getattr(lib, name).restype = ci
         lib.vig_bigla_fwd_host.argtypes = [vp] * 6 + [ci] * 5 + [cf, ci, vp]
         lib.vig_bigla_fwd_host.restype = ci
         lib.vig_status_string.argtypes = [ci]
@@ -204,6 +207,16 @@ def vig_bigla_bwd(q, k, v, log_alpha_fwd, log_alpha_bwd, d_out, dq, dk, dv, dlog
         raise ValueError("all tensors of one call share a dtype")
     _check(getattr(load(), name)(*(t.data_ptr() for t in ts), *_dims(q, v), _stream(stream)), name)
     return dq, dk, dv, dlog_alpha_fwd, dlog_alpha_bwd
+
+
+def vig_gate_prep_bwd(g_fwd, g_bwd, dlog_alpha_fwd, dlog_alpha_bwd, dg_fwd, dg_bwd, tau=16.0, stream=None):
+    """Gradient through the gate preparation: dg = dlog_alpha * sigmoid(-g) / tau, both directions."""
+    ts = (g_fwd, g_bwd, dlog_alpha_fwd, dlog_alpha_bwd, dg_fwd, dg_bwd)
+    _dev(*ts)
+    name = _by_dtype(g_fwd, "vig_gate_prep_bwd")
+    B, H, L, dk = g_fwd.shape
+    _check(getattr(load(), name)(*(t.data_ptr() for t in ts), B, H, L, dk, float(tau), _stream(stream)), name)
+    return dg_fwd, dg_bwd
 
 
 def vig_dwconv3x3(x, w, bias, out, stream=None):

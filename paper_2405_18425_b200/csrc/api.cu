@@ -273,6 +273,20 @@ static int gate_prep_impl(const void* g_f, const void* g_b, void* la_f, void* la
     return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
 }
 
+template <typename T>
+static int gate_prep_bwd_impl(const void* g_f, const void* g_b, const void* d_f, const void* d_b, void* o_f, void* o_b, int B, int H, int L,
+                              int dk, float tau, cudaStream_t stream) {
+    bool empty;
+    int st = check_gate_args(g_f, g_b, o_f, o_b, B, H, L, dk, tau, &empty);
+    if (st != VIG_OK) return st;
+    if (!d_f || !d_b) return VIG_ERR_NULL_POINTER;
+    if (!aligned16(d_f) || !aligned16(d_b)) return VIG_ERR_MISALIGNED;
+    if (empty) return VIG_OK;
+    const long long n = (long long)B * H * L * dk;
+    cudaError_t e = launch_gate_prep_bwd<T>((const T*)g_f, (const T*)g_b, (const T*)d_f, (const T*)d_b, (T*)o_f, (T*)o_b, n, tau, stream);
+    return e == cudaSuccess ? VIG_OK : VIG_ERR_CUDA;
+}
+
 // ---- host-buffer path: per device, two copy streams and the events that order them with the caller's stream -------
 constexpr int kHostSlices = 4;
 struct HostPath {
@@ -385,6 +399,16 @@ int vig_gate_prep_bf16(const void* g_fwd, const void* g_bwd, void* log_alpha_fwd
 int vig_gate_prep_f32(const void* g_fwd, const void* g_bwd, void* log_alpha_fwd, void* log_alpha_bwd, int B, int H,
                       int L, int dk, float tau, void* stream) {
     return gate_prep_impl<float>(g_fwd, g_bwd, log_alpha_fwd, log_alpha_bwd, B, H, L, dk, tau, (cudaStream_t)stream);
+}
+
+int vig_gate_prep_bwd_bf16(const void* g_fwd, const void* g_bwd, const void* dlog_alpha_fwd, const void* dlog_alpha_bwd, void* dg_fwd,
+                           void* dg_bwd, int B, int H, int L, int dk, float tau, void* stream) {
+    return gate_prep_bwd_impl<__nv_bfloat16>(g_fwd, g_bwd, dlog_alpha_fwd, dlog_alpha_bwd, dg_fwd, dg_bwd, B, H, L, dk, tau, (cudaStream_t)stream);
+}
+
+int vig_gate_prep_bwd_f32(const void* g_fwd, const void* g_bwd, const void* dlog_alpha_fwd, const void* dlog_alpha_bwd, void* dg_fwd,
+                          void* dg_bwd, int B, int H, int L, int dk, float tau, void* stream) {
+    return gate_prep_bwd_impl<float>(g_fwd, g_bwd, dlog_alpha_fwd, dlog_alpha_bwd, dg_fwd, dg_bwd, B, H, L, dk, tau, (cudaStream_t)stream);
 }
 
 int vig_bigla_fwd_host(const void* q, const void* k, const void* v, const void* g_fwd, const void* g_bwd, void* out,

@@ -72,6 +72,76 @@ __global__ void __launch_bounds__(256) gate_prep_kernel(const T* g_f, const T* g
     }
 }
 
+// Gradient through the gate preparation: dg = dlog alpha * sigmoid(-g) / tau (d/dg log sigmoid(g) = 1 - sigmoid(g)),
+// in fp32; exp only of non-positive numbers.
+__device__ __forceinline__ float gate_grad_of(float g, float d, float inv_tau) {
+    const float e = __expf(-fabsf(g));
+    return d * (g >= 0.f ? e : 1.f) / (1.f + e) * inv_tau;
+}
+
+// 16-byte vector body with a scalar tail; blockIdx.y picks the direction.
+template <typename T>
+__global__ void __launch_bounds__(256) gate_prep_bwd_kernel(const T* g_f, const T* g_b, const T* d_f, const T* d_b, T* o_f, T* o_b, long long n,
+                                                            float inv_tau) {
+    // no __restrict__: the output may be the incoming gradient's buffer
+    pdl_launch_dependents();
+    pdl_wait();
+    const T* g = blockIdx.y == 0 ? g_f : g_b;
+    const T* d = blockIdx.y == 0 ? d_f : d_b;
+    T* o = blockIdx.y == 0 ? o_f : o_b;
+    constexpr int V = 16 / sizeof(T);
+    const long long nvec = n / V, stride = (long long)gridDim.x * blockDim.x;
+    for (long long x = (long long)blockIdx.x * blockDim.x + threadIdx.x; x < nvec; x += stride) {
+        uint4 rg = reinterpret_cast<const uint4*>(g)[x], rd = reinterpret_cast<const uint4*>(d)[x];
+        if constexpr (sizeof(T) == 4) {
+            float *fg = reinterpret_cast<float*>(&rg), *fd = reinterpret_cast<float*>(&rd);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) fd[e] = gate_grad_of(fg[e], fd[e], inv_tau);
+        } else {
+            __nv_bfloat162 *hg = reinterpret_cast<__nv_bfloat162*>(&rg), *hd = reinterpret_cast<__nv_bfloat162*>(&rd);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 a = __bfloat1622float2(hg[e]), b = __bfloat1622float2(hd[e]);
+                hd[e] = __floats2bfloat162_rn(gate_grad_of(a.x, b.x, inv_tau), gate_grad_of(a.y, b.y, inv_tau));
+            }
+        }
+        reinterpret_cast<uint4*>(o)[x] = rd;
+    }
+    for (long long x = nvec * V + (long long)blockIdx.x * blockDim.x + threadIdx.x; x < n; x += stride) {
+        if constexpr (sizeof(T) == 4) o[x] = gate_grad_of(g[x], d[x], inv_tau);
+        else o[x] = __float2bfloat16_rn(gate_grad_of(__bfloat162float(g[x]), __bfloat162float(d[x]), inv_tau));
+    }
+}
+
+static cudaError_t gate_blocks(long long n, int vec, long long* blocks) {
+    static std::atomic<int> sms_of[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    int sms = sms_of[dev].load(std::memory_order_relaxed);
+    if (sms == 0) {
+        const cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        sms_of[dev].store(sms, std::memory_order_relaxed);
+    }
+    long long b = (n / vec + 255) / 256;
+    if (b < 1) b = 1;
+    if (b > 4LL * sms) b = 4LL * sms;
+    *blocks = b;
+    return cudaSuccess;
+}
+
+template <typename T>
+cudaError_t launch_gate_prep_bwd(const T* g_f, const T* g_b, const T* d_f, const T* d_b, T* o_f, T* o_b, long long n, float tau,
+                                 cudaStream_t stream) {
+    long long blocks = 1;
+    const cudaError_t e = gate_blocks(n, 16 / (int)sizeof(T), &blocks);
+    if (e != cudaSuccess) return e;
+    const cudaError_t le = launch_pdl(gate_prep_bwd_kernel<T>, dim3((unsigned)blocks, 2), dim3(256), 0, stream, g_f, g_b, d_f, d_b, o_f, o_b, n,
+                                      1.0f / tau);
+    count_launch();
+    return le != cudaSuccess ? le : cudaGetLastError();
+}
+
 template <typename T>
 cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long long n, float tau,
                              cudaStream_t stream) {
@@ -95,6 +165,10 @@ cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long 
     return le != cudaSuccess ? le : cudaGetLastError();
 }
 
+template cudaError_t launch_gate_prep_bwd<float>(const float*, const float*, const float*, const float*, float*, float*, long long, float,
+                                                 cudaStream_t);
+template cudaError_t launch_gate_prep_bwd<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, const __nv_bfloat16*,
+                                                         const __nv_bfloat16*, __nv_bfloat16*, __nv_bfloat16*, long long, float, cudaStream_t);
 template cudaError_t launch_gate_prep<float>(const float*, const float*, float*, float*, long long, float,
                                              cudaStream_t);
 template cudaError_t launch_gate_prep<__nv_bfloat16>(const __nv_bfloat16*, const __nv_bfloat16*, __nv_bfloat16*,

@@ -27,6 +27,10 @@ cudaError_t launch_recurrence(const T* q, const T* k, const T* v, const T* la_f,
 template <typename T>
 cudaError_t launch_gate_prep(const T* g_f, const T* g_b, T* la_f, T* la_b, long long n, float tau,
                              cudaStream_t stream);
+// dg = dlog alpha * sigmoid(-g) / tau, both directions in one launch (the outputs may be the incoming gradients' buffers)
+template <typename T>
+cudaError_t launch_gate_prep_bwd(const T* g_f, const T* g_b, const T* d_f, const T* d_b, T* o_f, T* o_b, long long n, float tau,
+                                 cudaStream_t stream);
 
 // ---- bf16 tensor-core path: dispatch over the tcgen05 kernels (defined with the entry points) ----
 bool tc_supported(int dk, int dv);

@@ -114,3 +114,23 @@ def test_gradient_entry_point_validates_arguments():
     assert lib.vig_bigla_bwd_bf16(*args, 1, 1, 8, 200, 32, None) == -3          # head size beyond the kernel's
     assert lib.vig_bigla_bwd_bf16(*args, 0, 1, 8, 16, 32, None) == 0            # empty
     assert vig.vig_kernel_launch_count() - before == launched
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("shape", [(2, 3, 196, 32), (1, 1, 1, 8), (1, 2, 5, 3), (3, 1, 33, 20)])
+def test_gate_prep_gradient_matches_oracle(oracle, dtype, shape):
+    """dg = dlog_alpha * sigmoid(-g) / tau against the oracle, vector body and scalar tail, separately and in place."""
+    r = np.random.default_rng(sum(shape))
+    g = [synth.store(r.standard_normal(shape) * 3, dtype) for _ in range(2)]
+    d = [synth.store(r.standard_normal(shape), dtype) for _ in range(2)]
+    f = lambda a: synth.stored_to_f64(a, dtype)
+    tg = [to_device(a, dtype) for a in g]
+    td = [to_device(a, dtype) for a in d]
+    out = [torch.full_like(t, float("nan")) for t in td]
+    vig.vig_gate_prep_bwd(tg[0], tg[1], td[0], td[1], out[0], out[1], 16.0)
+    vig.vig_gate_prep_bwd(tg[0], tg[1], td[0], td[1], td[0], td[1], 16.0)   # in place over the incoming gradients
+    torch.cuda.synchronize()
+    for x in range(2):
+        ref = oracle.gate_prep_bwd(f(g[x]), f(d[x]), 16.0)
+        assert rel_err(device_to_f64(out[x], dtype), ref) <= (2.0 ** -8 if dtype == "bf16" else 1e-6)
+        np.testing.assert_array_equal(to_stored(out[x], dtype), to_stored(td[x], dtype))
