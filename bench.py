@@ -437,7 +437,11 @@ def run_gpu(args, cfg):
     line["bwd_step"] = dict(_summary(bwd_ms), step="vig_bigla_bwd_bf16", algorithmic_bytes=bwd_bytes,
                             achieved_gbs=bwd_bytes / (bwd_us * 1e-6) / 1e9, frac_hbm=bwd_bytes / (bwd_us * 1e-6) / 1e9 / peak,
                             walk_fp32_tflops=walk_flops / (bwd_us * 1e-6) / 1e12, frac_alu=walk_flops / (bwd_us * 1e-6) / alu_peak,
-                            tokens_per_s=tokens_per_step / (bwd_us * 1e-6))
+                            tokens_per_s=tokens_per_step / (bwd_us * 1e-6),
+                            roofline={"bound": "alu", "achieved": walk_flops / (bwd_us * 1e-6) / 1e12, "peak": alu_peak / 1e12,
+                                      "unit": "TFLOP/s", "frac": walk_flops / (bwd_us * 1e-6) / alu_peak, "traffic": None,
+                                      "peak_source": "SMs x 128 fp32 lanes x 2 x 1.965 GHz",
+                                      "kernel": "bigla_bwd_kernel (the walks' flops over the time of the whole call)"})
 
     if rank == 0:
         # ---- end to end through the host-buffer entry point (H2D + kernels + D2H in the timed region) ----
