@@ -134,3 +134,24 @@ def test_gate_prep_gradient_matches_oracle(oracle, dtype, shape):
         ref = oracle.gate_prep_bwd(f(g[x]), f(d[x]), 16.0)
         assert rel_err(device_to_f64(out[x], dtype), ref) <= (2.0 ** -8 if dtype == "bf16" else 1e-6)
         np.testing.assert_array_equal(to_stored(out[x], dtype), to_stored(td[x], dtype))
+
+
+@pytest.mark.parametrize("B,H,L,dk,dv", [(16, 4, 196, 32, 64), (2, 2, 1100, 24, 48), (3, 2, 300, 40, 72)])
+def test_gradient_is_bitwise_reproducible(B, H, L, dk, dv):
+    """Whole units, segmented walks and the element-wise staging: four calls on the same inputs give the same bytes (the
+    asynchronous staging and the in-place results leave no room for a race that this would not show sooner or later)."""
+    cfg, x = random_problem(4400 + L, B, H, L, dk, dv, "bf16", gate_mean=1.0)
+    d = {n: to_device(a, "bf16") for n, a in x.items()}
+    d["d_out"] = to_device(synth.make_grad_input(cfg), "bf16")
+    la_f, la_b = torch.empty_like(d["g_fwd"]), torch.empty_like(d["g_bwd"])
+    vig.vig_gate_prep_bf16(d["g_fwd"], d["g_bwd"], la_f, la_b, cfg.tau)
+    first = None
+    for _ in range(4):
+        outs = [torch.full_like(d[n], float("nan")) for n in ("q", "k", "v", "q", "q")]
+        vig.vig_bigla_bwd(d["q"], d["k"], d["v"], la_f, la_b, d["d_out"], *outs)
+        torch.cuda.synchronize()
+        got = [to_stored(o, "bf16") for o in outs]
+        if first is None:
+            first = got
+        for a, b in zip(first, got):
+            np.testing.assert_array_equal(a, b)
